@@ -1,0 +1,138 @@
+/*
+ * regenvc_attn.h -- C ABI of the B200 (sm_100a) fused 3D-RoPE attention library.
+ *
+ * The operation is the attention step of the paper's real-time decoder: every
+ * block of the four-step diffusion transformer runs exact, non-causal
+ * multi-head softmax attention over the whole flattened T x H x W latent-token
+ * sequence of a 25-frame window (Sec. 3.5: after the Ulysses exchange each
+ * device "computes exact attention over the full sequence for a subset of
+ * heads"; here that is done for all heads on one GPU with no sharding), and
+ * cross-attention of the same queries to the short, precomputed text/image
+ * conditioning key/value tensors (Sec. 3.9).  The backbone's 3D rotary
+ * position embedding is applied to queries and keys inside the call.
+ *
+ * Conventions common to every entry point
+ *   - Tensors are bf16, contiguous, layout [tokens, n_heads, head_dim];
+ *     token n of a T x H x W grid is n = (t*H + y)*W + x.  Batch is 1; a
+ *     caller with several windows loops (or gives each GPU its own window).
+ *   - head_dim must be 128.  Rotary pairs are the adjacent elements
+ *     (2j, 2j+1); head_dim is split 44/42/42 over (t, y, x), each axis a 1-D
+ *     rotary embedding of its own width with frequencies theta^(-2i/width).
+ *     Scores are scaled by 1/sqrt(head_dim).  No mask.
+ *   - Arithmetic: inputs are widened exactly; rotated Q/K, V and the softmax
+ *     probabilities are rounded to fp16 tensor-core operands (inputs must
+ *     therefore be finite with |x| <= 65504); all accumulation is fp32; the
+ *     output is rounded once to bf16 (nearest even).  NaN/Inf inputs give
+ *     unspecified results.
+ *   - Pointers marked "device" must be valid on the current CUDA device and
+ *     16-byte aligned; the caller owns them, and the library neither frees
+ *     nor keeps them beyond the stream-ordered work of the call.
+ *   - Device entry points are asynchronous on `stream` (a cudaStream_t cast
+ *     to void*, NULL = legacy default stream) and never synchronise the host
+ *     once the workspace and the rotary table for the shape exist.
+ *   - Errors are return codes only; arguments are validated before any CUDA
+ *     work is enqueued, and a failing call enqueues nothing.
+ *   - There is no CPU path: on a machine without an sm_100 GPU every compute
+ *     entry point returns REGENVC_ERR_UNSUPPORTED or REGENVC_ERR_CUDA.
+ *   - Calls on one stream are ordered as usual.  Calls that overlap on the
+ *     GPU (different streams) must not share a workspace: give each stream
+ *     its own with regenvc_set_workspace() from the thread that launches on
+ *     it (the setting is per host thread), or serialise them.
+ */
+#ifndef REGENVC_ATTN_H
+#define REGENVC_ATTN_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    REGENVC_OK = 0,
+    REGENVC_ERR_NULL_POINTER = 1,
+    REGENVC_ERR_BAD_SHAPE = 2,   /* a dimension < 1 or a size that overflows */
+    REGENVC_ERR_UNSUPPORTED = 3, /* head_dim != 128, theta <= 0, device is not sm_100 */
+    REGENVC_ERR_MISALIGNED = 4,  /* a device pointer is not 16-byte aligned */
+    REGENVC_ERR_ALIASING = 5,    /* out overlaps q, k or v */
+    REGENVC_ERR_CUDA = 6,        /* a CUDA call failed: see regenvc_last_cuda_error() */
+    REGENVC_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired (sticky device status) */
+    REGENVC_ERR_WORKSPACE = 8,   /* caller-supplied workspace too small or misaligned */
+    REGENVC_ERR_RANGE = 9        /* an input exceeded the fp16 operand range (sticky device status) */
+} regenvc_status;
+
+/*
+ * Self-attention with fused 3D RoPE (Sec. 3.5; rotary convention as above).
+ *   q, k, v : device, bf16 [T*H*W, n_heads, head_dim]           (read only)
+ *   out     : device, bf16 [T*H*W, n_heads, head_dim]           (written; must not overlap q/k/v)
+ *   rope_theta : rotary base (> 0), 10000 for the paper's backbone
+ * out[n, a, :] = sum_m softmax_m( <R(n) q[n,a], R(m) k[m,a]> / sqrt(head_dim) ) v[m,a, :]
+ * Returns REGENVC_OK once the work is enqueued on `stream`.
+ */
+int regenvc_attn_forward(const void* q, const void* k, const void* v, void* out,
+                         int T, int H, int W, int n_heads, int head_dim,
+                         float rope_theta, void* stream);
+
+/*
+ * Cross-attention to a short conditioning sequence (Sec. 3.9: keys/values of
+ * the 512 text tokens or the 257 image tokens, computed once per sequence).
+ * No rotation, no mask.
+ *   q, out : device, bf16 [n_q, n_heads, head_dim]
+ *   k, v   : device, bf16 [n_kv, n_heads, head_dim]
+ */
+int regenvc_cross_attn_forward(const void* q, const void* k, const void* v, void* out,
+                               int n_q, int n_kv, int n_heads, int head_dim, void* stream);
+
+/*
+ * The same two operations for callers whose tensors live in HOST memory
+ * (pinned memory gives asynchronous copies; pageable memory works but is
+ * staged by the driver).  The call copies q, k, v to device staging buffers
+ * that the library owns and reuses, runs the device path, copies the result
+ * back into `out` and waits for `stream` before returning.
+ */
+int regenvc_attn_forward_host(const void* q, const void* k, const void* v, void* out,
+                              int T, int H, int W, int n_heads, int head_dim,
+                              float rope_theta, void* stream);
+int regenvc_cross_attn_forward_host(const void* q, const void* k, const void* v, void* out,
+                                    int n_q, int n_kv, int n_heads, int head_dim, void* stream);
+
+/*
+ * Scratch memory.  Each call first rewrites the keys and values into
+ * tensor-core operand form in a device workspace:
+ *   K' : fp16 [n_heads][n_kv_pad][128]   rotated (self) or converted (cross) keys
+ *   V't: fp16 [n_heads][128][n_kv_pad]   values, transposed so that keys are contiguous
+ * with n_kv_pad = n_kv rounded up to a multiple of 128 (padding is zero),
+ * K' first, V't directly after it.  regenvc_workspace_bytes() returns the
+ * size this needs (0 for invalid arguments).  By default the library keeps
+ * one workspace per device and host thread and grows it on demand with
+ * cudaMalloc (which synchronises: do a warm-up call before capturing a CUDA
+ * graph).  regenvc_set_workspace() makes the calling host thread use a
+ * caller-owned device buffer instead (256-byte aligned; NULL/0 returns to the
+ * internal one); a call that needs more than `bytes` then fails with
+ * REGENVC_ERR_WORKSPACE.
+ */
+size_t regenvc_workspace_bytes(int n_kv, int n_heads, int head_dim);
+int regenvc_set_workspace(void* dev_ptr, size_t bytes);
+
+/*
+ * Waits for `stream` and reports the sticky device-side status of the current
+ * device in *status_out: REGENVC_OK, REGENVC_ERR_TIMEOUT (a kernel gave up on
+ * a bounded wait; its output is invalid) or REGENVC_ERR_RANGE.  The status is
+ * cleared by the call.  Returns REGENVC_OK or the error of the query itself.
+ */
+int regenvc_device_status(void* stream, int* status_out);
+
+const char* regenvc_status_string(int status);
+/* Text of the last failing CUDA call on this host thread ("" if none). */
+const char* regenvc_last_cuda_error(void);
+const char* regenvc_version(void);
+/* Number of kernels the library has launched from this process (all threads). */
+unsigned long long regenvc_kernel_launch_count(void);
+/* Frees cached rotary tables, staging buffers and internal workspaces of every
+ * device.  No library work may be in flight. */
+void regenvc_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REGENVC_ATTN_H */

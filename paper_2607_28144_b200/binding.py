@@ -1,0 +1,180 @@
+"""Thin ctypes binding of the C ABI declared in ``include/regenvc_attn.h``.
+
+Argument marshalling only: every step of the attention path runs in the CUDA
+library.  PyTorch supplies device memory and streams.  If the shared library
+is missing the first call raises; there is no CPU or library fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libregenvc_attn.so")
+
+OK, ERR_NULL_POINTER, ERR_BAD_SHAPE, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_ALIASING, ERR_CUDA, ERR_TIMEOUT, \
+    ERR_WORKSPACE, ERR_RANGE = range(10)
+
+EXPORTS = [
+    "regenvc_attn_forward", "regenvc_cross_attn_forward", "regenvc_attn_forward_host",
+    "regenvc_cross_attn_forward_host", "regenvc_workspace_bytes", "regenvc_set_workspace",
+    "regenvc_device_status", "regenvc_status_string", "regenvc_last_cuda_error", "regenvc_version",
+    "regenvc_kernel_launch_count", "regenvc_shutdown",
+]
+
+_lib = None
+
+
+class RegenvcError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"regenvc status {code}: {text}")
+        self.code = code
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the CUDA shared library (built by ``python -m paper_2607_28144_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_28144_b200.build` "
+                           "(there is no fallback path)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, f32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    L.regenvc_attn_forward.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, vp]
+    L.regenvc_attn_forward.restype = i32
+    L.regenvc_cross_attn_forward.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+    L.regenvc_cross_attn_forward.restype = i32
+    L.regenvc_attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, vp]
+    L.regenvc_attn_forward_host.restype = i32
+    L.regenvc_cross_attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+    L.regenvc_cross_attn_forward_host.restype = i32
+    L.regenvc_workspace_bytes.argtypes = [i32, i32, i32]
+    L.regenvc_workspace_bytes.restype = sz
+    L.regenvc_set_workspace.argtypes = [vp, sz]
+    L.regenvc_set_workspace.restype = i32
+    L.regenvc_device_status.argtypes = [vp, ctypes.POINTER(i32)]
+    L.regenvc_device_status.restype = i32
+    L.regenvc_status_string.argtypes = [i32]
+    L.regenvc_status_string.restype = ctypes.c_char_p
+    L.regenvc_last_cuda_error.argtypes = []
+    L.regenvc_last_cuda_error.restype = ctypes.c_char_p
+    L.regenvc_version.argtypes = []
+    L.regenvc_version.restype = ctypes.c_char_p
+    L.regenvc_kernel_launch_count.argtypes = []
+    L.regenvc_kernel_launch_count.restype = ctypes.c_ulonglong
+    L.regenvc_shutdown.argtypes = []
+    L.regenvc_shutdown.restype = None
+    _lib = L
+    return L
+
+
+def status_string(code: int) -> str:
+    return lib().regenvc_status_string(code).decode()
+
+
+def _check(code: int):
+    if code != OK:
+        text = status_string(code)
+        if code == ERR_CUDA:
+            text += ": " + lib().regenvc_last_cuda_error().decode()
+        raise RegenvcError(code, text)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dev_bf16(t: torch.Tensor, name: str):
+    if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or t.dim() != 3:
+        raise TypeError(f"{name} must be a contiguous CUDA bf16 tensor [tokens, heads, head_dim]")
+
+
+def _host_bf16(t: torch.Tensor, name: str):
+    if t.dtype != torch.bfloat16 or t.is_cuda or not t.is_contiguous() or t.dim() != 3:
+        raise TypeError(f"{name} must be a contiguous CPU bf16 tensor [tokens, heads, head_dim]")
+
+
+def regenvc_attn_forward(q, k, v, out, T: int, H: int, W: int, rope_theta: float = 10000.0, stream=None):
+    """Self-attention with fused 3D RoPE on device tensors; asynchronous on ``stream``."""
+    for t, nm in ((q, "q"), (k, "k"), (v, "v"), (out, "out")):
+        _dev_bf16(t, nm)
+    n, h, d = q.shape
+    if n != T * H * W or k.shape != q.shape or v.shape != q.shape or out.shape != q.shape:
+        raise ValueError("q, k, v, out must all be [T*H*W, heads, head_dim]")
+    _check(lib().regenvc_attn_forward(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), T, H, W, h, d,
+                                      float(rope_theta), _stream(stream)))
+    return out
+
+
+def regenvc_cross_attn_forward(q, k, v, out, stream=None):
+    """Cross-attention of q [n_q, h, d] to k, v [n_kv, h, d] on device tensors."""
+    for t, nm in ((q, "q"), (k, "k"), (v, "v"), (out, "out")):
+        _dev_bf16(t, nm)
+    n_q, h, d = q.shape
+    n_kv = k.shape[0]
+    if k.shape != (n_kv, h, d) or v.shape != k.shape or out.shape != q.shape:
+        raise ValueError("shape mismatch")
+    _check(lib().regenvc_cross_attn_forward(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), n_q, n_kv, h, d,
+                                            _stream(stream)))
+    return out
+
+
+def regenvc_attn_forward_host(q, k, v, out, T: int, H: int, W: int, rope_theta: float = 10000.0, stream=None):
+    """Same operation with all four tensors in host memory (copies inside the call; returns when done)."""
+    for t, nm in ((q, "q"), (k, "k"), (v, "v"), (out, "out")):
+        _host_bf16(t, nm)
+    n, h, d = q.shape
+    if n != T * H * W or k.shape != q.shape or v.shape != q.shape or out.shape != q.shape:
+        raise ValueError("q, k, v, out must all be [T*H*W, heads, head_dim]")
+    _check(lib().regenvc_attn_forward_host(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), T, H, W, h, d,
+                                           float(rope_theta), _stream(stream)))
+    return out
+
+
+def regenvc_cross_attn_forward_host(q, k, v, out, stream=None):
+    for t, nm in ((q, "q"), (k, "k"), (v, "v"), (out, "out")):
+        _host_bf16(t, nm)
+    n_q, h, d = q.shape
+    n_kv = k.shape[0]
+    if k.shape != (n_kv, h, d) or v.shape != k.shape or out.shape != q.shape:
+        raise ValueError("shape mismatch")
+    _check(lib().regenvc_cross_attn_forward_host(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), n_q, n_kv,
+                                                 h, d, _stream(stream)))
+    return out
+
+
+def regenvc_workspace_bytes(n_kv: int, n_heads: int, head_dim: int = 128) -> int:
+    return int(lib().regenvc_workspace_bytes(n_kv, n_heads, head_dim))
+
+
+def regenvc_set_workspace(buf: Optional[torch.Tensor]):
+    """Use ``buf`` (a CUDA uint8 tensor the caller keeps alive) as this thread's workspace; None resets."""
+    if buf is None:
+        _check(lib().regenvc_set_workspace(None, 0))
+    else:
+        _check(lib().regenvc_set_workspace(buf.data_ptr(), buf.numel() * buf.element_size()))
+
+
+def regenvc_device_status(stream=None) -> int:
+    """Waits for ``stream`` and returns (then clears) the sticky device status."""
+    st = ctypes.c_int(0)
+    _check(lib().regenvc_device_status(_stream(stream), ctypes.byref(st)))
+    return st.value
+
+
+def regenvc_version() -> str:
+    return lib().regenvc_version().decode()
+
+
+def regenvc_kernel_launch_count() -> int:
+    return int(lib().regenvc_kernel_launch_count())
+
+
+def regenvc_shutdown():
+    lib().regenvc_shutdown()

@@ -1,0 +1,417 @@
+// Host side of the C ABI: argument validation, per-device state (status word,
+// rotary tables, workspaces, staging buffers), TMA tensor maps and launches.
+#include <atomic>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <string>
+#include <thread>
+#include <vector>
+
+#include "../../include/regenvc_attn.h"
+#include "common.cuh"
+
+namespace regenvc {
+cudaError_t configure_attn_serial();
+cudaError_t launch_attn_serial(const CUtensorMap&, const CUtensorMap&, const AttnParams&, cudaStream_t);
+cudaError_t configure_attn_pipelined();
+cudaError_t launch_attn_pipelined(const CUtensorMap&, const CUtensorMap&, const AttnParams&, cudaStream_t);
+}  // namespace regenvc
+
+namespace {
+
+using namespace regenvc;
+
+struct Buf {
+    void* ptr = nullptr;
+    size_t bytes = 0;
+};
+struct RopeEntry {
+    int T, H, W;
+    float theta;
+    float2* dev;
+};
+struct DeviceState {
+    bool checked = false, supported = false;
+    int* status = nullptr;
+    int sm_count = 0;
+    std::vector<RopeEntry> ropes;
+    std::map<std::thread::id, Buf> workspace;
+    std::map<std::thread::id, std::vector<Buf>> staging;  // q, k, v, out
+};
+
+std::mutex g_mu;
+std::map<int, DeviceState> g_dev;
+std::atomic<unsigned long long> g_launches{0};
+thread_local std::string tl_cuda_error;
+thread_local Buf tl_user_ws;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+int cuda_fail(cudaError_t e, const char* what) {
+    tl_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+    (void)cudaGetLastError();
+    return REGENVC_ERR_CUDA;
+}
+#define CUDA_TRY(expr)                                   \
+    do {                                                 \
+        cudaError_t e_ = (expr);                         \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #expr); \
+    } while (0)
+
+bool serial_kernel_requested() {
+    static const bool serial = [] {
+        const char* e = std::getenv("REGENVC_KERNEL");
+        return e && std::strcmp(e, "serial") == 0;
+    }();
+    return serial;
+}
+
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + nb && b0 < a0 + na;
+}
+
+// Validation common to both operations; no CUDA call is made here.
+int validate(const void* q, const void* k, const void* v, void* out, long long n_q, long long n_kv, int n_heads,
+             int head_dim, bool device_ptrs) {
+    if (!q || !k || !v || !out) return REGENVC_ERR_NULL_POINTER;
+    if (n_q < 1 || n_kv < 1 || n_heads < 1 || head_dim < 1) return REGENVC_ERR_BAD_SHAPE;
+    // token * head row indices (including the padded key rows of the workspace) are 32-bit in the TMA coordinates
+    const long long kv_pad = (n_kv + kTile - 1) / kTile * kTile;
+    if (n_q > (1ll << 30) || n_kv > (1ll << 30) || n_heads > 65535 || kv_pad * n_heads >= (1ll << 31) ||
+        n_q * n_heads >= (1ll << 31))
+        return REGENVC_ERR_BAD_SHAPE;
+    if (head_dim != kHeadDim) return REGENVC_ERR_UNSUPPORTED;
+    if (device_ptrs) {
+        if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15) return REGENVC_ERR_MISALIGNED;
+    }
+    const size_t qb = (size_t)n_q * n_heads * head_dim * 2, kb = (size_t)n_kv * n_heads * head_dim * 2;
+    if (overlaps(out, qb, q, qb) || overlaps(out, qb, k, kb) || overlaps(out, qb, v, kb)) return REGENVC_ERR_ALIASING;
+    return REGENVC_OK;
+}
+
+int device_state(int* dev_out, DeviceState** st_out) {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    DeviceState& st = g_dev[dev];
+    if (!st.checked) {
+        int major = 0;
+        CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        CUDA_TRY(cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev));
+        st.supported = (major == 10);
+        if (st.supported) {
+            if (!g_encode) {
+                void* fn = nullptr;
+                cudaDriverEntryPointQueryResult qres;
+                CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+                if (!fn || qres != cudaDriverEntryPointSuccess) {
+                    tl_cuda_error = "cuTensorMapEncodeTiled is not available in this driver";
+                    return REGENVC_ERR_CUDA;
+                }
+                g_encode = (EncodeTiledFn)fn;
+            }
+            CUDA_TRY(configure_attn_serial());
+            CUDA_TRY(configure_attn_pipelined());
+            CUDA_TRY(cudaMalloc(&st.status, sizeof(int)));
+            CUDA_TRY(cudaMemset(st.status, 0, sizeof(int)));
+        }
+        st.checked = true;
+    }
+    *dev_out = dev;
+    *st_out = &st;
+    return st.supported ? REGENVC_OK : REGENVC_ERR_UNSUPPORTED;
+}
+
+int grow(Buf& b, size_t bytes) {
+    if (b.bytes >= bytes) return REGENVC_OK;
+    if (b.ptr) CUDA_TRY(cudaFree(b.ptr));  // waits for work that may still use it
+    b.ptr = nullptr;
+    b.bytes = 0;
+    CUDA_TRY(cudaMalloc(&b.ptr, bytes));
+    b.bytes = bytes;
+    return REGENVC_OK;
+}
+
+// cos/sin of every (axis position, pair) in double precision, stored as float2.
+int rope_table(DeviceState& st, int T, int H, int W, float theta, const float2** out) {
+    for (const RopeEntry& e : st.ropes)
+        if (e.T == T && e.H == H && e.W == W && e.theta == theta) {
+            *out = e.dev;
+            return REGENVC_OK;
+        }
+    std::vector<float2> host((size_t)T * kPairsT + (size_t)H * kPairsY + (size_t)W * kPairsX);
+    size_t at = 0;
+    const int extent[3] = {T, H, W};
+    const int pairs[3] = {kPairsT, kPairsY, kPairsX};
+    for (int axis = 0; axis < 3; ++axis)
+        for (int pos = 0; pos < extent[axis]; ++pos)
+            for (int i = 0; i < pairs[axis]; ++i) {
+                const double freq = std::pow((double)theta, -(double)i / (double)pairs[axis]);
+                const double ang = (double)pos * freq;
+                host[at++] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+            }
+    float2* dev = nullptr;
+    CUDA_TRY(cudaMalloc(&dev, host.size() * sizeof(float2)));
+    cudaError_t e = cudaMemcpy(dev, host.data(), host.size() * sizeof(float2), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        cudaFree(dev);
+        return cuda_fail(e, "cudaMemcpy(rope table)");
+    }
+    st.ropes.push_back(RopeEntry{T, H, W, theta, dev});
+    *out = dev;
+    return REGENVC_OK;
+}
+
+int make_tmap(CUtensorMap* m, void* base, uint64_t inner, uint64_t outer, uint64_t row_bytes) {
+    const cuuint64_t gdim[2] = {inner, outer};
+    const cuuint64_t gstride[1] = {row_bytes};
+    const cuuint32_t box[2] = {64, 128};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, gdim, gstride, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        tl_cuda_error = "cuTensorMapEncodeTiled failed with CUresult " + std::to_string((int)r);
+        return REGENVC_ERR_CUDA;
+    }
+    return REGENVC_OK;
+}
+
+size_t workspace_need(long long n_kv, int n_heads) {
+    const size_t kv_pad = (size_t)((n_kv + kTile - 1) / kTile * kTile);
+    return 2 * (size_t)n_heads * kv_pad * kHeadDim * sizeof(__half);
+}
+
+// Enqueues the two kernels.  Arguments are already validated; pointers are device pointers.
+int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int n_kv, int n_heads, bool rope, int T,
+            int H, int W, float theta, cudaStream_t stream) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev = 0;
+    DeviceState* st = nullptr;
+    int rc = device_state(&dev, &st);
+    if (rc != REGENVC_OK) return rc;
+
+    const size_t need = workspace_need(n_kv, n_heads);
+    void* ws = nullptr;
+    if (tl_user_ws.ptr) {
+        if (tl_user_ws.bytes < need) return REGENVC_ERR_WORKSPACE;
+        ws = tl_user_ws.ptr;
+    } else {
+        Buf& b = st->workspace[std::this_thread::get_id()];
+        rc = grow(b, need);
+        if (rc != REGENVC_OK) return rc;
+        ws = b.ptr;
+    }
+    const int kv_pad = round_up(n_kv, kTile);
+    __half* kp = reinterpret_cast<__half*>(ws);
+    __half* vt = kp + (size_t)n_heads * kv_pad * kHeadDim;
+
+    RopeGrid grid{nullptr, T, H, W};
+    if (rope) {
+        rc = rope_table(*st, T, H, W, theta, &grid.tab);
+        if (rc != REGENVC_OK) return rc;
+    }
+
+    CUtensorMap tmap_k, tmap_v;
+    rc = make_tmap(&tmap_k, kp, kHeadDim, (uint64_t)n_heads * kv_pad, kHeadDim * sizeof(__half));
+    if (rc != REGENVC_OK) return rc;
+    rc = make_tmap(&tmap_v, vt, (uint64_t)kv_pad, (uint64_t)n_heads * kHeadDim, (uint64_t)kv_pad * sizeof(__half));
+    if (rc != REGENVC_OK) return rc;
+
+    PrepParams pp;
+    pp.k = reinterpret_cast<const __nv_bfloat16*>(k);
+    pp.v = reinterpret_cast<const __nv_bfloat16*>(v);
+    pp.kp = kp;
+    pp.vt = vt;
+    pp.n_kv = n_kv;
+    pp.n_kv_pad = kv_pad;
+    pp.h = n_heads;
+    pp.rope = rope ? 1 : 0;
+    pp.grid = grid;
+    pp.status = st->status;
+    CUDA_TRY(launch_prep_kv(pp, stream));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+
+    AttnParams ap;
+    ap.q = reinterpret_cast<const __nv_bfloat16*>(q);
+    ap.out = reinterpret_cast<__nv_bfloat16*>(out);
+    ap.n_q = n_q;
+    ap.n_kv = n_kv;
+    ap.n_kv_pad = kv_pad;
+    ap.h = n_heads;
+    ap.rope = rope ? 1 : 0;
+    ap.grid = grid;
+    ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)kHeadDim));
+    ap.status = st->status;
+    ap.sm_count = st->sm_count;
+    if (serial_kernel_requested())
+        CUDA_TRY(launch_attn_serial(tmap_k, tmap_v, ap, stream));
+    else
+        CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, ap, stream));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return REGENVC_OK;
+}
+
+// Host-buffer variant: stage in, run, stage out, wait.
+int run_host(const void* q, const void* k, const void* v, void* out, int n_q, int n_kv, int n_heads, bool rope, int T,
+             int H, int W, float theta, cudaStream_t stream) {
+    const size_t qb = (size_t)n_q * n_heads * kHeadDim * 2, kb = (size_t)n_kv * n_heads * kHeadDim * 2;
+    void *dq, *dk, *dv, *dout;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        int dev = 0;
+        DeviceState* st = nullptr;
+        int rc = device_state(&dev, &st);
+        if (rc != REGENVC_OK) return rc;
+        std::vector<Buf>& s = st->staging[std::this_thread::get_id()];
+        s.resize(4);
+        const size_t need[4] = {qb, kb, kb, qb};
+        for (int i = 0; i < 4; ++i) {
+            rc = grow(s[i], need[i]);
+            if (rc != REGENVC_OK) return rc;
+        }
+        dq = s[0].ptr; dk = s[1].ptr; dv = s[2].ptr; dout = s[3].ptr;
+    }
+    CUDA_TRY(cudaMemcpyAsync(dq, q, qb, cudaMemcpyHostToDevice, stream));
+    CUDA_TRY(cudaMemcpyAsync(dk, k, kb, cudaMemcpyHostToDevice, stream));
+    CUDA_TRY(cudaMemcpyAsync(dv, v, kb, cudaMemcpyHostToDevice, stream));
+    int rc = enqueue(dq, dk, dv, dout, n_q, n_kv, n_heads, rope, T, H, W, theta, stream);
+    if (rc != REGENVC_OK) return rc;
+    CUDA_TRY(cudaMemcpyAsync(out, dout, qb, cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    return REGENVC_OK;
+}
+
+int check_self_args(int T, int H, int W, float theta, long long* n_out) {
+    if (T < 1 || H < 1 || W < 1) return REGENVC_ERR_BAD_SHAPE;
+    const long long n = (long long)T * H * W;
+    if (n > (1ll << 30)) return REGENVC_ERR_BAD_SHAPE;
+    *n_out = n;
+    (void)theta;
+    return REGENVC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int regenvc_attn_forward(const void* q, const void* k, const void* v, void* out, int T, int H, int W, int n_heads,
+                         int head_dim, float rope_theta, void* stream) {
+    if (!q || !k || !v || !out) return REGENVC_ERR_NULL_POINTER;
+    long long n = 0;
+    int rc = check_self_args(T, H, W, rope_theta, &n);
+    if (rc != REGENVC_OK) return rc;
+    rc = validate(q, k, v, out, n, n, n_heads, head_dim, true);
+    if (rc != REGENVC_OK) return rc;
+    if (!(rope_theta > 0.0f) || !std::isfinite(rope_theta)) return REGENVC_ERR_UNSUPPORTED;
+    return enqueue(q, k, v, out, (int)n, (int)n, n_heads, true, T, H, W, rope_theta, (cudaStream_t)stream);
+}
+
+int regenvc_cross_attn_forward(const void* q, const void* k, const void* v, void* out, int n_q, int n_kv, int n_heads,
+                               int head_dim, void* stream) {
+    int rc = validate(q, k, v, out, n_q, n_kv, n_heads, head_dim, true);
+    if (rc != REGENVC_OK) return rc;
+    return enqueue(q, k, v, out, n_q, n_kv, n_heads, false, 1, 1, 1, 1.0f, (cudaStream_t)stream);
+}
+
+int regenvc_attn_forward_host(const void* q, const void* k, const void* v, void* out, int T, int H, int W, int n_heads,
+                              int head_dim, float rope_theta, void* stream) {
+    if (!q || !k || !v || !out) return REGENVC_ERR_NULL_POINTER;
+    long long n = 0;
+    int rc = check_self_args(T, H, W, rope_theta, &n);
+    if (rc != REGENVC_OK) return rc;
+    rc = validate(q, k, v, out, n, n, n_heads, head_dim, false);
+    if (rc != REGENVC_OK) return rc;
+    if (!(rope_theta > 0.0f) || !std::isfinite(rope_theta)) return REGENVC_ERR_UNSUPPORTED;
+    return run_host(q, k, v, out, (int)n, (int)n, n_heads, true, T, H, W, rope_theta, (cudaStream_t)stream);
+}
+
+int regenvc_cross_attn_forward_host(const void* q, const void* k, const void* v, void* out, int n_q, int n_kv,
+                                    int n_heads, int head_dim, void* stream) {
+    int rc = validate(q, k, v, out, n_q, n_kv, n_heads, head_dim, false);
+    if (rc != REGENVC_OK) return rc;
+    return run_host(q, k, v, out, n_q, n_kv, n_heads, false, 1, 1, 1, 1.0f, (cudaStream_t)stream);
+}
+
+size_t regenvc_workspace_bytes(int n_kv, int n_heads, int head_dim) {
+    if (n_kv < 1 || n_heads < 1 || head_dim != kHeadDim) return 0;
+    return workspace_need(n_kv, n_heads);
+}
+
+int regenvc_set_workspace(void* dev_ptr, size_t bytes) {
+    if (!dev_ptr || bytes == 0) {
+        tl_user_ws = Buf{};
+        return REGENVC_OK;
+    }
+    if ((uintptr_t)dev_ptr & 255) return REGENVC_ERR_WORKSPACE;
+    tl_user_ws.ptr = dev_ptr;
+    tl_user_ws.bytes = bytes;
+    return REGENVC_OK;
+}
+
+int regenvc_device_status(void* stream, int* status_out) {
+    if (!status_out) return REGENVC_ERR_NULL_POINTER;
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev = 0;
+    DeviceState* st = nullptr;
+    int rc = device_state(&dev, &st);
+    if (rc != REGENVC_OK) return rc;
+    CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    int h = 0;
+    CUDA_TRY(cudaMemcpy(&h, st->status, sizeof(int), cudaMemcpyDeviceToHost));
+    if (h != 0) CUDA_TRY(cudaMemset(st->status, 0, sizeof(int)));
+    *status_out = h;
+    return REGENVC_OK;
+}
+
+const char* regenvc_status_string(int status) {
+    switch (status) {
+        case REGENVC_OK: return "ok";
+        case REGENVC_ERR_NULL_POINTER: return "null pointer";
+        case REGENVC_ERR_BAD_SHAPE: return "bad shape";
+        case REGENVC_ERR_UNSUPPORTED: return "unsupported (head_dim must be 128, theta > 0, device sm_100)";
+        case REGENVC_ERR_MISALIGNED: return "device pointer not 16-byte aligned";
+        case REGENVC_ERR_ALIASING: return "out overlaps an input";
+        case REGENVC_ERR_CUDA: return "CUDA call failed";
+        case REGENVC_ERR_TIMEOUT: return "device-side bounded wait expired";
+        case REGENVC_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case REGENVC_ERR_RANGE: return "input outside the fp16 operand range";
+        default: return "unknown status";
+    }
+}
+
+const char* regenvc_last_cuda_error(void) { return tl_cuda_error.c_str(); }
+
+const char* regenvc_version(void) { return "regenvc-attn 0.1 (sm_100a)"; }
+
+unsigned long long regenvc_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+void regenvc_shutdown(void) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        g_dev.clear();
+        return;
+    }
+    for (auto& kv : g_dev) {
+        if (cudaSetDevice(kv.first) != cudaSuccess) continue;
+        DeviceState& st = kv.second;
+        if (st.status) cudaFree(st.status);
+        for (RopeEntry& e : st.ropes) cudaFree(e.dev);
+        for (auto& w : st.workspace) cudaFree(w.second.ptr);
+        for (auto& s : st.staging)
+            for (Buf& b : s.second) cudaFree(b.ptr);
+    }
+    g_dev.clear();
+    cudaSetDevice(prev);
+    (void)cudaGetLastError();
+}
+
+}  // extern "C"

@@ -1,0 +1,213 @@
+"""GPU parity: the CUDA path, called through the C ABI binding, against the
+fp64 oracle on the same seeded inputs (element by element on small shapes)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_28144_b200 import binding, synth
+from parity_util import assert_parity, errors, f64, hull_check, run_gpu_cross, run_gpu_self
+
+pytestmark = pytest.mark.gpu
+
+D = 128
+
+
+def _rand(rng, n, h, scale=1.0):
+    return synth.from_f32(rng.standard_normal((n, h, D)) * scale)
+
+
+def _self_case(T, H, W, h, seed, scale=1.0, theta=10000.0):
+    rng = np.random.default_rng(seed)
+    N = T * H * W
+    q, k, v = _rand(rng, N, h, scale), _rand(rng, N, h, scale), _rand(rng, N, h, scale)
+    gpu = f64(run_gpu_self(q, k, v, T, H, W, theta))
+    ref = oracle.self_attention(synth.bits(q), synth.bits(k), synth.bits(v), T, H, W, theta)
+    hull_check(gpu, f64(v))
+    return assert_parity(gpu, ref, float(v.float().abs().max()), f"self {T}x{H}x{W} h={h}")
+
+
+def test_workspace_holds_rotated_keys_and_transposed_values():
+    """The preparation pass: K' equals the oracle's rotated keys to fp16 rounding; V't is V transposed exactly."""
+    T, H, W, h = 3, 5, 11, 3
+    N = T * H * W
+    n_pad = (N + 127) // 128 * 128
+    rng = np.random.default_rng(5)
+    q, k, v = _rand(rng, N, h), _rand(rng, N, h), _rand(rng, N, h)
+    nbytes = binding.regenvc_workspace_bytes(N, h)
+    assert nbytes == 2 * h * n_pad * D * 2
+    ws = torch.full((nbytes,), 0xFF, dtype=torch.uint8, device="cuda:0")
+    binding.regenvc_set_workspace(ws)
+    try:
+        run_gpu_self(q, k, v, T, H, W)
+    finally:
+        binding.regenvc_set_workspace(None)
+    halves = ws.view(torch.float16).cpu()
+    kp = halves[: h * n_pad * D].view(h, n_pad, D).double().numpy()
+    vt = halves[h * n_pad * D:].view(h, D, n_pad).double().numpy()
+    for a in range(h):
+        ref = oracle.rope_rotate_head(synth.bits(k), T, H, W, a)
+        np.testing.assert_allclose(kp[a, :N], ref, rtol=2 ** -10, atol=1e-6)
+        assert (kp[a, N:] == 0).all() and (vt[a, :, N:] == 0).all()
+        np.testing.assert_array_equal(vt[a, :, :N], f64(v)[:, a, :].T)
+
+
+@pytest.mark.parametrize("grid,h", [
+    ((1, 1, 1), 1), ((1, 1, 2), 1), ((2, 3, 4), 2), ((1, 1, 127), 1), ((1, 1, 129), 2), ((127, 1, 1), 1),
+    ((1, 127, 1), 1), ((3, 5, 7), 3), ((2, 8, 8), 2), ((1, 11, 12), 1), ((1, 15, 17), 2), ((1, 16, 16), 3),
+    ((1, 1, 257), 1), ((3, 7, 13), 2), ((2, 13, 17), 3), ((5, 9, 11), 2),
+])
+def test_self_attention_small_shapes(grid, h):
+    T, H, W = grid
+    _self_case(T, H, W, h, seed=1000 + T * H * W + h)
+
+
+def test_self_attention_window_256x256():
+    w = synth.WORKLOADS["window_256x256"]
+    q, k, v = synth.self_inputs(w)
+    gpu = f64(run_gpu_self(q, k, v, w.T, w.H, w.W, w.theta))
+    ref = oracle.self_attention(synth.bits(q), synth.bits(k), synth.bits(v), w.T, w.H, w.W, w.theta)
+    hull_check(gpu, f64(v))
+    e = assert_parity(gpu, ref, float(v.float().abs().max()), w.name)
+    for a in range(w.n_heads):  # per head, to localise a bad head
+        assert errors(gpu[:, a], ref[:, a], float(v.float().abs().max()))["mre"] <= 2e-3
+    print("window_256x256", e)
+
+
+def test_tiny_workload_against_brute_force_too():
+    w = synth.WORKLOADS["tiny"]
+    q, k, v = synth.self_inputs(w)
+    gpu = f64(run_gpu_self(q, k, v, w.T, w.H, w.W, w.theta))
+    maxv = float(v.float().abs().max())
+    for a in range(w.n_heads):
+        assert_parity(gpu[:, a], oracle.brute_force(synth.bits(q), synth.bits(k), synth.bits(v), w.T, w.H, w.W, a),
+                      maxv, "tiny vs brute force")
+    assert_parity(gpu, oracle.self_attention(synth.bits(q), synth.bits(k), synth.bits(v), w.T, w.H, w.W), maxv, "tiny")
+
+
+@pytest.mark.parametrize("scale", [0.5, 2.0])
+def test_self_attention_score_range(scale):
+    # q, k, v scaled: score standard deviation 0.25 and 4 (softmax from nearly flat to peaked)
+    _self_case(2, 13, 17, 2, seed=77, scale=scale)
+
+
+@pytest.mark.parametrize("theta", [1.0, 100.0, 1e6])
+def test_self_attention_other_theta(theta):
+    _self_case(3, 6, 9, 2, seed=78, theta=theta)
+
+
+@pytest.mark.parametrize("n_q,n_kv,h", [
+    (1, 1, 1), (1, 7, 2), (129, 127, 1), (129, 128, 2), (129, 129, 1), (1, 257, 2), (300, 257, 3), (1792, 512, 2),
+    (129, 769, 2), (1792, 257, 12), (513, 512, 12),
+])
+def test_cross_attention(n_q, n_kv, h):
+    rng = np.random.default_rng(2000 + n_q + n_kv + h)
+    q, k, v = _rand(rng, n_q, h), _rand(rng, n_kv, h), _rand(rng, n_kv, h)
+    gpu = f64(run_gpu_cross(q, k, v))
+    ref = oracle.cross_attention(synth.bits(q), synth.bits(k), synth.bits(v))
+    hull_check(gpu, f64(v))
+    assert_parity(gpu, ref, float(v.float().abs().max()), f"cross {n_q}x{n_kv} h={h}")
+
+
+# ---------------------------------------------------------------- structured inputs that localise bugs
+def test_zero_queries_give_column_mean_everywhere():
+    T, H, W, h = 2, 11, 13, 2
+    N = T * H * W
+    rng = np.random.default_rng(31)
+    k, v = _rand(rng, N, h), _rand(rng, N, h)
+    q = torch.zeros_like(k)
+    gpu = f64(run_gpu_self(q, k, v, T, H, W))
+    mean = f64(v).mean(axis=0)
+    assert np.abs(gpu - mean[None]).max() <= 2 ** -8 * np.abs(mean).max() + 1e-3
+
+
+def test_constant_value_rows_come_back_exactly():
+    T, H, W, h = 1, 9, 31, 2
+    N = T * H * W
+    rng = np.random.default_rng(32)
+    q, k = _rand(rng, N, h, 2.0), _rand(rng, N, h, 2.0)
+    crow = _rand(rng, 1, h)
+    v = crow.expand(N, h, D).contiguous()
+    gpu = f64(run_gpu_self(q, k, v, T, H, W))
+    # sum_m p_m c / sum_m p_m = c up to fp32 accumulation and one bf16 rounding
+    np.testing.assert_allclose(gpu, np.broadcast_to(f64(crow), gpu.shape), rtol=2 ** -8, atol=1e-6)
+
+
+def test_position_probe_values():
+    """v_m = (t, y, x, 1, m mod 128 one-hot ...): the output is the attention-weighted mean position and the
+    probability mass per key residue; exposes a wrong token map, a dropped key tile or a wrong tail mask."""
+    T, H, W, h = 3, 7, 15, 1
+    N = T * H * W
+    rng = np.random.default_rng(33)
+    q, k = _rand(rng, N, h, 1.5), _rand(rng, N, h, 1.5)
+    n = np.arange(N)
+    v = np.zeros((N, h, D), dtype=np.float32)
+    v[:, 0, 0], v[:, 0, 1], v[:, 0, 2], v[:, 0, 3] = n // (H * W), (n // W) % H, n % W, 1.0
+    v[n, 0, 4 + (n % 124)] = 1.0
+    v = synth.from_f32(v)
+    gpu = f64(run_gpu_self(q, k, v, T, H, W))
+    ref = oracle.self_attention(synth.bits(q), synth.bits(k), synth.bits(v), T, H, W)
+    np.testing.assert_allclose(gpu[:, 0, 3], 1.0, rtol=2 ** -8)
+    np.testing.assert_allclose(gpu[:, 0, 4:].sum(axis=1), 1.0, rtol=1e-2)
+    assert_parity(gpu, ref, float(v.float().abs().max()), "position probe")
+
+
+def test_dominating_key_and_large_scores():
+    T, H, W, h = 1, 5, 60, 1
+    N = T * H * W
+    rng = np.random.default_rng(34)
+    q, k, v = _rand(rng, N, h), _rand(rng, N, h), _rand(rng, N, h)
+    gpu = f64(run_gpu_self(q, (k.float() * 6).to(torch.bfloat16), v, T, H, W))
+    ref = oracle.self_attention(synth.bits(q), synth.bits((k.float() * 6).to(torch.bfloat16)), synth.bits(v), T, H, W)
+    assert_parity(gpu, ref, float(v.float().abs().max()), "peaked softmax")
+
+
+def test_heads_are_independent_on_the_gpu():
+    T, H, W, h = 2, 9, 10, 4
+    N = T * H * W
+    rng = np.random.default_rng(35)
+    q, k, v = _rand(rng, N, h), _rand(rng, N, h), _rand(rng, N, h)
+    full = run_gpu_self(q, k, v, T, H, W)
+    sub = run_gpu_self(q[:, 1:3].contiguous(), k[:, 1:3].contiguous(), v[:, 1:3].contiguous(), T, H, W)
+    assert torch.equal(full[:, 1:3], sub)
+
+
+def test_repeated_calls_are_bitwise_reproducible_and_host_variant_matches():
+    w = synth.WORKLOADS["tiny"]
+    q, k, v = synth.self_inputs(w)
+    a = run_gpu_self(q, k, v, w.T, w.H, w.W)
+    b = run_gpu_self(q, k, v, w.T, w.H, w.W)
+    assert torch.equal(a, b)
+    out = torch.empty_like(q).pin_memory()
+    binding.regenvc_attn_forward_host(q.pin_memory(), k.pin_memory(), v.pin_memory(), out, w.T, w.H, w.W)
+    assert torch.equal(out, a)
+    kc, vc = synth.cross_inputs(synth.WORKLOADS["window_480x832"], 257)
+    kc, vc = kc[:, :2].contiguous(), vc[:, :2].contiguous()
+    c = run_gpu_cross(q, kc, vc)
+    outc = torch.empty_like(q)
+    binding.regenvc_cross_attn_forward_host(q, kc, vc, outc)
+    assert torch.equal(outc, c)
+
+
+def test_out_of_range_input_sets_the_range_status():
+    q = torch.zeros((4, 1, D), dtype=torch.bfloat16)
+    k = torch.zeros((4, 1, D), dtype=torch.bfloat16)
+    k[2, 0, 5] = 1e6  # beyond fp16
+    dev = torch.device("cuda:0")
+    out = torch.empty((4, 1, D), dtype=torch.bfloat16, device=dev)
+    binding.regenvc_cross_attn_forward(q.to(dev), k.to(dev), k.to(dev), out)
+    assert binding.regenvc_device_status() == binding.ERR_RANGE
+    assert binding.regenvc_device_status() == 0  # cleared by the query
+
+
+def test_workspace_too_small_is_rejected():
+    dev = torch.device("cuda:0")
+    t = torch.zeros((200, 1, D), dtype=torch.bfloat16, device=dev)
+    ws = torch.empty((1024,), dtype=torch.uint8, device=dev)
+    binding.regenvc_set_workspace(ws)
+    try:
+        with pytest.raises(binding.RegenvcError) as ei:
+            binding.regenvc_cross_attn_forward(t, t, t, torch.empty_like(t))
+        assert ei.value.code == binding.ERR_WORKSPACE
+    finally:
+        binding.regenvc_set_workspace(None)
