@@ -122,6 +122,16 @@ int regenvc_set_workspace(void* dev_ptr, size_t bytes);
  */
 int regenvc_device_status(void* stream, int* status_out);
 
+/*
+ * Profiling aid: selects which of the two kernels later calls from this host
+ * thread enqueue.  Bit 0 = key/value preparation pass, bit 1 = attention
+ * kernel; the default is 3 (both).  With bit 0 clear the workspace must still
+ * hold the prepared operands of the same k, v and shape (from an earlier full
+ * call), which lets a benchmark time the attention kernel alone.  Returns
+ * REGENVC_ERR_BAD_SHAPE for a mask outside 1..3.
+ */
+int regenvc_debug_set_phases(int mask);
+
 const char* regenvc_status_string(int status);
 /* Text of the last failing CUDA call on this host thread ("" if none). */
 const char* regenvc_last_cuda_error(void);

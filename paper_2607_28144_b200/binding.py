@@ -22,7 +22,7 @@ EXPORTS = [
     "regenvc_attn_forward", "regenvc_cross_attn_forward", "regenvc_attn_forward_host",
     "regenvc_cross_attn_forward_host", "regenvc_workspace_bytes", "regenvc_set_workspace",
     "regenvc_device_status", "regenvc_status_string", "regenvc_last_cuda_error", "regenvc_version",
-    "regenvc_kernel_launch_count", "regenvc_shutdown",
+    "regenvc_kernel_launch_count", "regenvc_shutdown", "regenvc_debug_set_phases",
 ]
 
 _lib = None
@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
     L.regenvc_version.restype = ctypes.c_char_p
     L.regenvc_kernel_launch_count.argtypes = []
     L.regenvc_kernel_launch_count.restype = ctypes.c_ulonglong
+    L.regenvc_debug_set_phases.argtypes = [i32]
+    L.regenvc_debug_set_phases.restype = i32
     L.regenvc_shutdown.argtypes = []
     L.regenvc_shutdown.restype = None
     _lib = L
@@ -174,6 +176,11 @@ def regenvc_version() -> str:
 
 def regenvc_kernel_launch_count() -> int:
     return int(lib().regenvc_kernel_launch_count())
+
+
+def regenvc_debug_set_phases(mask: int):
+    """Profiling aid: 1 = preparation pass only, 2 = attention kernel only, 3 = both (default)."""
+    _check(lib().regenvc_debug_set_phases(mask))
 
 
 def regenvc_shutdown():

@@ -47,6 +47,7 @@ std::map<int, DeviceState> g_dev;
 std::atomic<unsigned long long> g_launches{0};
 thread_local std::string tl_cuda_error;
 thread_local Buf tl_user_ws;
+thread_local int tl_phases = 3;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -235,8 +236,11 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     pp.rope = rope ? 1 : 0;
     pp.grid = grid;
     pp.status = st->status;
-    CUDA_TRY(launch_prep_kv(pp, stream));
-    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (tl_phases & 1) {
+        CUDA_TRY(launch_prep_kv(pp, stream));
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    if (!(tl_phases & 2)) return REGENVC_OK;
 
     AttnParams ap;
     ap.q = reinterpret_cast<const __nv_bfloat16*>(q);
@@ -367,6 +371,12 @@ int regenvc_device_status(void* stream, int* status_out) {
     CUDA_TRY(cudaMemcpy(&h, st->status, sizeof(int), cudaMemcpyDeviceToHost));
     if (h != 0) CUDA_TRY(cudaMemset(st->status, 0, sizeof(int)));
     *status_out = h;
+    return REGENVC_OK;
+}
+
+int regenvc_debug_set_phases(int mask) {
+    if (mask < 1 || mask > 3) return REGENVC_ERR_BAD_SHAPE;
+    tl_phases = mask;
     return REGENVC_OK;
 }
 
