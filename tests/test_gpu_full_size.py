@@ -1,0 +1,76 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration bench.py times: sampled query rows
+against the fp64 oracle (rows are independent, so a sampled row is checked exactly as a full run would), plus
+closed forms that cover every row at any size."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_28144_b200 import binding, synth
+from parity_util import MRE_LIMIT, assert_parity, errors, f64, hull_check, run_gpu_cross, run_gpu_self
+
+pytestmark = pytest.mark.gpu
+
+
+def _heads_to_check(w, scales):
+    if w.n_heads <= 12:
+        return list(range(w.n_heads))
+    picks = {0, w.n_heads - 1, w.n_heads // 2, 7, 13, 22}
+    if scales is not None:
+        picks.add(int(torch.argmin(scales)))
+        picks.add(int(torch.argmax(scales)))
+    return sorted(picks)[:8]
+
+
+@pytest.mark.parametrize("name", ["window_480x832", "large_480x832_ref", "clip_77f"])
+def test_full_size_sampled_rows(name):
+    w = synth.WORKLOADS[name]
+    q, k, v = synth.self_inputs(w)
+    scales = synth.head_scales(w.seed, w.n_heads, *w.head_scale) if w.head_scale else None
+    gpu = run_gpu_self(q, k, v, w.T, w.H, w.W, w.theta)
+    rows = synth.sample_rows(w.n_tokens, w.H, w.W, seed=w.seed)
+    heads = _heads_to_check(w, scales)
+    qb, kb, vb = synth.bits(q), synth.bits(k), synth.bits(v)
+    max_v = float(v.float().abs().max())
+    got_all, ref_all = [], []
+    for a in heads:
+        ref = oracle.self_attn_head(qb, kb, vb, w.T, w.H, w.W, a, w.theta, rows=rows)
+        got = gpu[rows, a].double().numpy()
+        e = assert_parity(got, ref, max_v, f"{name} head {a}")
+        got_all.append(got)
+        ref_all.append(ref)
+    e = assert_parity(np.stack(got_all), np.stack(ref_all), max_v, name)
+    print(name, "rows", len(rows), "heads", heads, e)
+    # convex-hull property on every element of the full output
+    gv = gpu.float()
+    vmax, vmin = v.float().amax(dim=0), v.float().amin(dim=0)
+    assert torch.isfinite(gv).all()
+    assert (gv <= vmax + 0.02 * vmax.abs() + 1e-3).all() and (gv >= vmin - 0.02 * vmin.abs() - 1e-3).all()
+    # cross-attention of the same queries to the conditioning sequences
+    for n_kv in w.cross_kv:
+        kc, vc = synth.cross_inputs(w, n_kv)
+        gc = run_gpu_cross(q, kc, vc)
+        for a in heads[:4]:
+            ref = oracle.cross_attn_head(qb, synth.bits(kc), synth.bits(vc), a, rows=rows)
+            assert_parity(gc[rows, a].double().numpy(), ref, float(vc.float().abs().max()), f"{name} cross {n_kv} head {a}")
+
+
+def test_full_size_closed_forms_cover_every_row():
+    w = synth.WORKLOADS["window_480x832"]
+    q, k, v = synth.self_inputs(w)
+    # constant value rows: every output row equals that row whatever Q and K are
+    crow = v[:1]
+    gpu = run_gpu_self(q, k, crow.expand_as(v).contiguous(), w.T, w.H, w.W)
+    assert torch.allclose(gpu.float(), crow.float().expand_as(gpu), rtol=2 ** -8, atol=1e-6)
+    # zero queries: uniform softmax, every output row is the column mean of V (tests the tail mask: a key
+    # counted twice or a padded key counted once would shift the mean by 1/10920 of a value)
+    gpu = run_gpu_self(torch.zeros_like(q), k, v, w.T, w.H, w.W)
+    mean = v.double().mean(dim=0)
+    err = (gpu.double() - mean[None]).abs()
+    assert float(err.max()) <= 2 ** -8 * float(mean.abs().max()) + 2e-4
+    # residue one-hot values: out[n, c] is the probability mass of keys = c (mod 128); rows must sum to 1
+    vv = torch.zeros_like(v)
+    n = torch.arange(w.n_tokens)
+    vv[n, :, n % 128] = 1.0
+    gpu = run_gpu_self(q, k, vv, w.T, w.H, w.W)
+    assert torch.allclose(gpu.float().sum(dim=-1), torch.ones(w.n_tokens, w.n_heads), rtol=5e-3, atol=0)
