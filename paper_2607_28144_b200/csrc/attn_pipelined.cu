@@ -1,22 +1,26 @@
 // Pipelined, warp-specialised tcgen05 attention kernel for sm_100a.
 //
 // One CTA owns one head and two 128-row query tiles (256 query rows):
-//   warps 0-3  softmax group 0 (query tile 0): one thread per query row
-//   warps 4-7  softmax group 1 (query tile 1)
+//   warps 0-7  softmax: warp w works on TMEM lanes (query rows) 32*(w%4).. and on key columns
+//              64*(w/4)..+63 of every score tile, so two threads share a row; the eight warps take the
+//              score tiles of the two query tiles in turn (S0(j), S1(j), S0(j+1), ...)
 //   warp  8    UMMA issuer (one elected lane) and TMEM owner
 //   warp  9    TMA producer (one elected lane): streams K' and V't tiles
-// The two query tiles ping-pong: while a softmax group turns S_t into P_t the
-// tensor core runs the other tile's P.V and next Q.K^T.
+//   warps 10-11 idle (they complete the third warpgroup, which hands its registers to the softmax warps)
+// While the softmax warps turn S_t into P_t the tensor core runs the other tile's P.V and next Q.K^T.
 //
 // Tensor memory (512 columns x 128 lanes, fp32 cells):
-//   [0,128) S0  [128,256) S1  [256,384) O0  [384,512) O1 ; P_t (fp16) aliases the first 64 columns of S_t.
-// Shared memory: Q0, Q1 (32 KB each, rotated, fp16, 128B-swizzled K-major
-// blocks), then a ring of kStages 32 KB slots holding K'_0, V't_0, K'_1, ...
+//   [0,128) S0  [128,256) S1  [256,384) O0  [384,512) O1.  P_t (fp16, two keys per cell) aliases S_t:
+//   keys 0..63 in columns [0,32), keys 64..127 in columns [64,96) of S_t, i.e. each half-row thread writes
+//   its probabilities over score columns it has already read itself.
+// Shared memory: Q0, Q1 (32 KB each, rotated, fp16, 128B-swizzled K-major blocks), then a ring of kStages
+// 32 KB slots holding K'_0, V't_0, K'_1, ...
 //
-// Softmax keeps a running reference m (log2 domain) and row sum l per thread.
-// m is only raised when the tile maximum exceeds it by more than kRescaleGap
-// (probabilities then stay <= 2^kRescaleGap, well inside fp16/fp32 range), so
-// the rescale of the O accumulator in TMEM is rare after the first tiles.
+// Softmax keeps, per row, a reference m (log2 domain) and a row sum l.  m is only raised when a tile's
+// maximum exceeds it by more than kRescaleGap (probabilities stay <= 2^kRescaleGap, inside fp16 range), so
+// after the first tile the probabilities are formed directly against the reference of the earlier tiles,
+// chunk by chunk as the scores arrive; the two threads of a row exchange their half-row maxima through
+// shared memory once per tile, and the rescale of the O accumulator (with a redo of the tile) is rare.
 #include "common.cuh"
 #include "ptx.cuh"
 #include "q_tile.cuh"
@@ -25,15 +29,33 @@
 
 namespace regenvc {
 
+#ifdef REGENVC_TRACE
+// Bring-up instrumentation (never compiled into the shipped library): clock64 stamps of one CTA.
+__device__ long long g_trace[64 * 16];
+#define TRACE(j, slot)                                                                  \
+    do {                                                                                \
+        if (blockIdx.x == 3 && blockIdx.y == 0 && (j) >= 16 && (j) < 80)                \
+            g_trace[((j) - 16) * 16 + (slot)] = clock64();                              \
+    } while (0)
+#else
+#define TRACE(j, slot) do {} while (0)
+#endif
+
 namespace {
 
 constexpr int kStages = 4;                       // K/V ring slots (32 KB each)
 constexpr int kSoftmaxThreads = 256;
-constexpr int kThreads = kSoftmaxThreads + 64;   // + UMMA warp + TMA warp
+constexpr int kThreads = kSoftmaxThreads + 128;  // + one warpgroup holding the UMMA and TMA warps
+constexpr int kSoftmaxRegs = 232, kControlRegs = 40;  // 256 * 232 + 128 * 40 <= 64 K registers
 constexpr int kMmaWarp = 8, kTmaWarp = 9;
 constexpr float kRescaleGap = 8.0f;
+#ifndef REGENVC_POLY_MASK
+#define REGENVC_POLY_MASK 0x52
+#endif
+// bit i set: pair i of every eight probability pairs takes the polynomial 2^x instead of the MUFU
+constexpr uint32_t kPolyMask = REGENVC_POLY_MASK;
 constexpr uint32_t kIdesc = umma_idesc_f16_f32acc(128, 128);
-constexpr uint32_t kSmemBytes = (2 + kStages) * kTileBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr uint32_t kSmemBytes = (2 + kStages) * kTileBytes + 1024 /*align*/ + 256 /*barriers*/ + 6144 /*row exchange*/;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 struct Barriers {
@@ -48,18 +70,82 @@ struct Barriers {
 };
 static_assert(sizeof(Barriers) <= 256, "barrier block too large");
 
+// Values the two threads of a row hand each other: [parity][tile][half][row].
+struct RowExchange {
+    float v[2][2][2][kTile];
+    float l[2][2][kTile];  // row sums at the end: [tile][half][row]
+};
+
+// 2^x for a packed pair on the FMA/ALU pipes: x = n + f with n = round(x), f in [-0.5, 0.5];
+// 2^f by a degree-3 minimax polynomial (max relative error 7.5e-5, below fp16 rounding of P),
+// 2^n by adding n to the exponent field.  x is clamped at -125 so that the exponent cannot wrap.
+__device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
+    float x0, x1;
+    unpack2(x2, x0, x1);
+    x2 = pack2(fmaxf(x0, -125.0f), fmaxf(x1, -125.0f));
+    const float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+    const uint64_t r2 = add2(x2, pack2(kMagic, kMagic));
+    const uint64_t n2 = add2(r2, pack2(-kMagic, -kMagic));
+    const uint64_t f2 = add2(x2, mul2(n2, pack2(-1.0f, -1.0f)));
+    uint64_t q2 = fma2(f2, pack2(0.0551716685f, 0.0551716685f), pack2(0.242611125f, 0.242611125f));
+    q2 = fma2(q2, f2, pack2(0.693260968f, 0.693260968f));
+    q2 = fma2(q2, f2, pack2(0.999928057f, 0.999928057f));
+    float q0, q1, r0, r1;
+    unpack2(q2, q0, q1);
+    unpack2(r2, r0, r1);
+    q0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(r0) << 23));
+    q1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(r1) << 23));
+    return pack2(q0, q1);
+}
+
+// Named barrier over the eight softmax warps (barrier 0 is __syncthreads).
+__device__ __forceinline__ void softmax_barrier() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
+}
+
+// 32 scores of one row -> 16 packed fp16 probability pairs p = 2^(s * scale - m_ref).  The FMA is done on
+// packed fp32 pairs; pair c of every eight uses the polynomial when bit (c % 8) of kMask is set, the MUFU
+// otherwise, which splits the exponentials between the two pipes.  The fp32 probabilities are also added
+// into two packed partial row sums.
+template <uint32_t kMask>
+__device__ __forceinline__ void exp_chunk(const uint32_t* s, uint64_t scale2, uint64_t negm2, uint32_t* pr,
+                                          uint64_t& sum_a, uint64_t& sum_b) {
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        const uint64_t x2 = fma2(pack2(__uint_as_float(s[2 * c]), __uint_as_float(s[2 * c + 1])), scale2, negm2);
+        uint64_t p2;
+        if ((kMask >> (c & 7)) & 1u) {
+            p2 = exp2_poly2(x2);
+        } else {
+            float x0, x1;
+            unpack2(x2, x0, x1);
+            p2 = pack2(ex2_approx(x0), ex2_approx(x1));
+        }
+        if (c & 1) sum_b = add2(sum_b, p2);
+        else sum_a = add2(sum_a, p2);
+        float p0, p1;
+        unpack2(p2, p0, p1);
+        pr[c] = pack_f16x2(p0, p1);
+    }
+}
+
+// The eight K = 16 steps of one 128 x 128 x 128 product.  Descriptors differ only in the start-address
+// field: +2 (32 bytes) per K step inside a 128-byte row, +1024 (16 KB) for the second 64-element block.
 __device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint32_t sQ, uint32_t sK) {
+    const uint64_t a0 = umma_smem_desc_k_sw128(sQ), b0 = umma_smem_desc_k_sw128(sK);
 #pragma unroll
     for (int kk = 0; kk < 8; ++kk) {
-        const uint32_t off = (kk >> 2) * kBlockBytes + (kk & 3) * 32;
-        umma_ss(d_tmem, umma_smem_desc_k_sw128(sQ + off), umma_smem_desc_k_sw128(sK + off), kIdesc, kk > 0);
+        const uint64_t off = (kk >> 2) * (kBlockBytes >> 4) + (kk & 3) * 2;
+        umma_ss(d_tmem, a0 + off, b0 + off, kIdesc, kk > 0);
     }
 }
 __device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint32_t sV, bool accumulate) {
+    const uint64_t b0 = umma_smem_desc_k_sw128(sV);
 #pragma unroll
     for (int kk = 0; kk < 8; ++kk) {
-        const uint32_t off = (kk >> 2) * kBlockBytes + (kk & 3) * 32;
-        umma_ts(d_tmem, p_tmem + kk * 8, umma_smem_desc_k_sw128(sV + off), kIdesc, accumulate || kk > 0);
+        const uint64_t off = (kk >> 2) * (kBlockBytes >> 4) + (kk & 3) * 2;
+        // P: keys 0..63 at columns [0,32), keys 64..127 at columns [64,96) of the score tile
+        umma_ts(d_tmem, p_tmem + (kk >> 2) * 64 + (kk & 3) * 8, b0 + off, kIdesc, accumulate || kk > 0);
     }
 }
 
@@ -73,6 +159,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     uint8_t* sQ = base;                       // 2 tiles
     uint8_t* sKV = base + 2 * kTileBytes;     // ring
     Barriers* bar = reinterpret_cast<Barriers*>(base + (2 + kStages) * kTileBytes);
+    RowExchange* xch = reinterpret_cast<RowExchange*>(base + (2 + kStages) * kTileBytes + 256);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int head = blockIdx.y;
@@ -86,9 +173,9 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             mbar_init(smem_u32(&bar->kv_empty[s]), 1);
         }
         for (int t = 0; t < 2; ++t) {
-            mbar_init(smem_u32(&bar->q_full[t]), kSoftmaxThreads / 2);
+            mbar_init(smem_u32(&bar->q_full[t]), kSoftmaxThreads);
             mbar_init(smem_u32(&bar->s_full[t]), 1);
-            mbar_init(smem_u32(&bar->p_full[t]), kSoftmaxThreads / 2);
+            mbar_init(smem_u32(&bar->p_full[t]), kSoftmaxThreads);
             mbar_init(smem_u32(&bar->o_full[t]), 1);
         }
         bar->abort_flag = 0;
@@ -98,7 +185,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         tmem_alloc(smem_u32(&bar->tmem_base), 512);
         tmem_relinquish();
     }
-    if (warp == kTmaWarp && lane == 0) {
+    if (warp == kTmaWarp && elect_one()) {
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
     }
@@ -109,9 +196,11 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     const uint32_t tmem_base = bar->tmem_base;
     const WaitCtl ctl{&bar->abort_flag, p.status, kStatusTimeout, kWaitLimitNs};
 
-    if (warp == kTmaWarp) {
+    if (warp >= kMmaWarp) {
+      setmaxnreg_dec<kControlRegs>();
+      if (warp == kTmaWarp) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        if (elect_one()) {
             const int total = 2 * n_tiles;
             for (int i = 0; i < total; ++i) {
                 const int slot = i % kStages, round = i / kStages;
@@ -129,9 +218,9 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 }
             }
         }
-    } else if (warp == kMmaWarp) {
+      } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------ UMMA issuer
-        if (lane == 0) {
+        if (elect_one()) {
             const uint32_t sQ0 = smem_u32(sQ), sQ1 = smem_u32(sQ) + kTileBytes;
             const int n_active = tile1_active ? 2 : 1;
             bool ok = mbar_wait(smem_u32(&bar->q_full[0]), 0, ctl);
@@ -155,12 +244,15 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     ok = mbar_wait(smem_u32(&bar->p_full[t]), j & 1, ctl);
                     if (!ok) break;
                     tc_fence_after();
+                    TRACE(j, 12 + t * 2);
                     issue_pv(tmem_base + 256 + t * 128, tmem_base + t * 128, smem_u32(sKV + slot_v * kTileBytes), j > 0);
                     umma_commit(smem_u32(&bar->o_full[t]));
+                    TRACE(j, 5 + t * 6);
                     if (more) {
                         issue_qk(tmem_base + t * 128, t ? sQ1 : sQ0, smem_u32(sKV + slot_k * kTileBytes));
                         umma_commit(smem_u32(&bar->s_full[t]));
                     }
+                    TRACE(j, 13 + t * 2);
                 }
                 if (ok) {
                     umma_commit(smem_u32(&bar->kv_empty[slot_v]));
@@ -168,104 +260,146 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 }
             }
         }
+      }
     } else {
         // ------------------------------------------------------------ softmax groups
-        const int t = warp >> 2;                 // query tile of this group
-        const int row = tid & 127;               // row in the tile == TMEM lane
-        const int qt0 = q0 + t * kTile;
-        if (t == 0 || tile1_active) {
-            load_rotate_q_tile(p, head, qt0, sQ + t * kTileBytes, row, kSoftmaxThreads / 2);
+        setmaxnreg_inc<kSoftmaxRegs>();
+        const int half = warp >> 2;                      // which 64 key columns of a score row
+        const int row = (warp & 3) * 32 + lane;          // row in the tile == TMEM lane
+        const int n_active = tile1_active ? 2 : 1;
+        for (int t = 0; t < n_active; ++t) {
+            load_rotate_q_tile(p, head, q0 + t * kTile, sQ + t * kTileBytes, tid, kSoftmaxThreads);
             fence_proxy_async_smem();
             mbar_arrive(smem_u32(&bar->q_full[t]));
+        }
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const float scale = p.scale_log2;
+        const uint64_t scale2 = pack2(scale, scale);
+        float m_ref[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+        bool ok = true;  // false once a wait expired: keep the loop structure (named barriers) but skip the work
 
-            const uint32_t lane_base = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-            const uint32_t t_S = lane_base + t * 128, t_O = lane_base + 256 + t * 128;
-            const uint32_t s_full = smem_u32(&bar->s_full[t]), p_full = smem_u32(&bar->p_full[t]),
-                           o_full = smem_u32(&bar->o_full[t]);
-            const float scale = p.scale_log2;
-            float m_ref = 0.f, l_run = 0.f;
-            bool ok = true;
-
-            for (int j = 0; j < n_tiles; ++j) {
-                ok = mbar_wait(s_full, j & 1, ctl);
-                if (!ok) break;
+        for (int j = 0; j < n_tiles; ++j) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                if (t >= n_active) continue;
+                const uint32_t t_S = lane_base + t * 128 + half * 64, t_O = lane_base + 256 + t * 128 + half * 64;
+                if (tid == 0) TRACE(j, t * 6 + 0);
+                if (ok) ok = mbar_wait(smem_u32(&bar->s_full[t]), j & 1, ctl);
+                ok = __all_sync(0xffffffffu, ok);  // keep the warp-wide TMEM instructions below convergent
                 tc_fence_after();
-                uint32_t sr[128];
-                tmem_ld32(t_S + 0, sr + 0);
-                tmem_ld32(t_S + 32, sr + 32);
-                tmem_ld32(t_S + 64, sr + 64);
-                tmem_ld32(t_S + 96, sr + 96);
-                tmem_wait_ld();
-                if (j == n_tiles - 1) {
-                    const int valid = p.n_kv - j * kTile;  // columns >= valid are padding
+                if (tid == 0) TRACE(j, t * 6 + 1);
+                uint32_t sr[64];
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                const int valid = ((j == n_tiles - 1) ? p.n_kv - j * kTile : kTile) - half * 64;  // own columns >= valid are padding
+                uint64_t negm2 = pack2(-m_ref[t], -m_ref[t]);
+                uint64_t sum_a = 0, sum_b = 0;  // packed partial row sums
+                const bool stream = j > 0;
+                if (ok) {
+                    tmem_ld32(t_S, sr);
 #pragma unroll
-                    for (int c = 0; c < 128; ++c)
-                        if (c >= valid) sr[c] = 0xff800000u;  // -inf
-                }
-                float mx = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
-                const float m_tile = mx * scale;
-                bool raise = (j == 0) || (m_tile > m_ref + kRescaleGap);
-                if (j > 0 && __any_sync(0xffffffffu, raise)) {
-                    // some row of this warp moves its reference: rescale this warp's O rows and row sums
-                    ok = mbar_wait(o_full, (j - 1) & 1, ctl);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const float alpha = raise ? ex2_approx(m_ref - m_tile) : 1.0f;
-                    l_run *= alpha;
-#pragma unroll 1
-                    for (int cb = 0; cb < 4; ++cb) {
-                        uint32_t o[32];
-                        tmem_ld32(t_O + cb * 32, o);
+                    for (int cb = 0; cb < 2; ++cb) {
                         tmem_wait_ld();
+                        if (cb == 0) tmem_ld32(t_S + 32, sr + 32);
+                        if (valid < 64) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                        tmem_st32(t_O + cb * 32, o);
+                            for (int c = 0; c < 32; ++c)
+                                if (cb * 32 + c >= valid) sr[cb * 32 + c] = 0xff800000u;  // -inf
+                        }
+#pragma unroll
+                        for (int c = 0; c < 32; c += 8) {
+                            const uint32_t* x = sr + cb * 32 + c;
+                            mx0 = max3(mx0, __uint_as_float(x[0]), __uint_as_float(x[1]));
+                            mx1 = max3(mx1, __uint_as_float(x[2]), __uint_as_float(x[3]));
+                            mx2 = max3(mx2, __uint_as_float(x[4]), __uint_as_float(x[5]));
+                            mx3 = max3(mx3, __uint_as_float(x[6]), __uint_as_float(x[7]));
+                        }
+                        if (stream) {
+                            uint32_t pr[16];
+                            exp_chunk<kPolyMask>(sr + cb * 32, scale2, negm2, pr, sum_a, sum_b);
+                            tmem_st16(t_S + cb * 16, pr);
+                        }
                     }
                 }
-                if (raise) m_ref = m_tile;
-                float rowsum = 0.f;
+                // the two threads of a row exchange their half-row maxima
+                const float mx_half = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                xch->v[j & 1][t][half][row] = mx_half;
+                softmax_barrier();
+                const float m_tile = fmaxf(mx_half, xch->v[j & 1][t][half ^ 1][row]) * scale;
+                if (tid == 0) TRACE(j, t * 6 + 2);
+                const bool raise = m_tile > m_ref[t] + kRescaleGap;  // always true on the first tile
+                const bool any_raise = __any_sync(0xffffffffu, raise);
+                if (ok && any_raise) {
+                    // some row of this warp moves its reference (the partner warp sees the same rows and takes
+                    // the same branch): rescale this thread's half of the O row and its row sum, then (re)compute
+                    // the probabilities of the tile against the new reference
+                    if (j > 0) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar->o_full[t]), (j - 1) & 1, ctl));
+                        tc_fence_after();
+                        const float alpha = raise ? ex2_approx(m_ref[t] - m_tile) : 1.0f;
+                        l_run[t] *= alpha;
+                        if (ok) {
+#pragma unroll 1
+                            for (int cb = 0; cb < 2; ++cb) {
+                                uint32_t o[32];
+                                tmem_ld32(t_O + cb * 32, o);
+                                tmem_wait_ld();
 #pragma unroll
-                for (int cb = 0; cb < 4; ++cb) {
-                    uint32_t pr[16];
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(sr[cb * 32 + 2 * c]), scale, -m_ref));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(sr[cb * 32 + 2 * c + 1]), scale, -m_ref));
-                        rowsum += p0 + p1;
-                        pr[c] = pack_f16x2(p0, p1);
+                                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                                tmem_st32(t_O + cb * 32, o);
+                            }
+                        }
                     }
-                    tmem_st16(t_S + cb * 16, pr);
+                    if (raise) m_ref[t] = m_tile;
+                    negm2 = pack2(-m_ref[t], -m_ref[t]);
+                    sum_a = 0;
+                    sum_b = 0;
+                    if (ok) {
+#pragma unroll
+                        for (int cb = 0; cb < 2; ++cb) {
+                            uint32_t pr[16];
+                            exp_chunk<kPolyMask>(sr + cb * 32, scale2, negm2, pr, sum_a, sum_b);
+                            tmem_st16(t_S + cb * 16, pr);
+                        }
+                    }
                 }
-                l_run += rowsum;
+                float s0, s1;
+                unpack2(add2(sum_a, sum_b), s0, s1);
+                l_run[t] += s0 + s1;
+                if (tid == 0) TRACE(j, t * 6 + 3);
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(p_full);
+                mbar_arrive(smem_u32(&bar->p_full[t]));
+                if (tid == 0) TRACE(j, t * 6 + 4);
             }
+        }
 
-            // epilogue: O / l -> bf16 -> out
-            if (ok) ok = mbar_wait(o_full, (n_tiles - 1) & 1, ctl);
-            if (ok) {
-                tc_fence_after();
-                const int n = qt0 + row;
-                const float inv_l = 1.0f / l_run;
+        // epilogue: O / l -> bf16 -> out; each thread owns 64 of the 128 output columns of its row
+        for (int t = 0; t < n_active; ++t) {
+            xch->l[t][half][row] = l_run[t];
+            softmax_barrier();
+            const float inv_l = 1.0f / (l_run[t] + xch->l[t][half ^ 1][row]);
+            if (ok) ok = mbar_wait(smem_u32(&bar->o_full[t]), (n_tiles - 1) & 1, ctl);
+            ok = __all_sync(0xffffffffu, ok);
+            tc_fence_after();
+            const int n = q0 + t * kTile + row;
+            const uint32_t t_O = lane_base + 256 + t * 128 + half * 64;
 #pragma unroll 1
-                for (int cb = 0; cb < 4; ++cb) {
-                    uint32_t o[32];
+            for (int cb = 0; cb < 2; ++cb) {
+                uint32_t o[32];
+                if (ok) {
                     tmem_ld32(t_O + cb * 32, o);
                     tmem_wait_ld();
-                    if (n < p.n_q) {
-                        uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)n * p.h + head) * kHeadDim + cb * 32);
+                }
+                if (ok && n < p.n_q) {
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)n * p.h + head) * kHeadDim + half * 64 + cb * 32);
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint4 w;
-                            w.x = pack_bf16x2(__uint_as_float(o[8 * c + 0]) * inv_l, __uint_as_float(o[8 * c + 1]) * inv_l);
-                            w.y = pack_bf16x2(__uint_as_float(o[8 * c + 2]) * inv_l, __uint_as_float(o[8 * c + 3]) * inv_l);
-                            w.z = pack_bf16x2(__uint_as_float(o[8 * c + 4]) * inv_l, __uint_as_float(o[8 * c + 5]) * inv_l);
-                            w.w = pack_bf16x2(__uint_as_float(o[8 * c + 6]) * inv_l, __uint_as_float(o[8 * c + 7]) * inv_l);
-                            dst[c] = w;
-                        }
+                    for (int c = 0; c < 4; ++c) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(o[8 * c + 0]) * inv_l, __uint_as_float(o[8 * c + 1]) * inv_l);
+                        w.y = pack_bf16x2(__uint_as_float(o[8 * c + 2]) * inv_l, __uint_as_float(o[8 * c + 3]) * inv_l);
+                        w.z = pack_bf16x2(__uint_as_float(o[8 * c + 4]) * inv_l, __uint_as_float(o[8 * c + 5]) * inv_l);
+                        w.w = pack_bf16x2(__uint_as_float(o[8 * c + 6]) * inv_l, __uint_as_float(o[8 * c + 7]) * inv_l);
+                        dst[c] = w;
                     }
                 }
             }
@@ -273,17 +407,26 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     }
 
     // ---------------------------------------------------------------- tear-down
+    __syncwarp();  // lanes that left a single-lane role loop rejoin before the warp-wide instructions below
     tc_fence_before();
     __syncthreads();
     if (warp == kMmaWarp) {
+        __syncwarp();
         if (bar->abort_flag) {
             // a wait expired: give copies and MMAs that may still be in flight time to land before TMEM is released
             const uint64_t t0 = global_timer_ns();
             while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
         }
+        __syncwarp();
         tmem_dealloc(tmem_base, 512);
     }
 }
+
+#ifdef REGENVC_TRACE
+extern "C" int regenvc_debug_read_trace(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(g_trace));
+}
+#endif
 
 cudaError_t configure_attn_pipelined() {
     return cudaFuncSetAttribute(attn_pipelined_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);

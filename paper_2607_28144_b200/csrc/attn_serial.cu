@@ -88,6 +88,7 @@ attn_serial_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             umma_commit(bar_s);
         }
         mbar_wait(bar_s, ph, ctl);
+        __syncwarp();
         tc_fence_after();
 
         // ---- softmax on this thread's row
@@ -147,6 +148,7 @@ attn_serial_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             umma_commit(bar_o);
         }
         mbar_wait(bar_o, ph, ctl);
+        __syncwarp();
         tc_fence_after();
     }
 
@@ -173,7 +175,10 @@ attn_serial_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem_base, 256);
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, 256);
+    }
 }
 
 cudaError_t configure_attn_serial() {
