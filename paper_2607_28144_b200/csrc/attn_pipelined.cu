@@ -16,11 +16,11 @@
 // Shared memory: Q0, Q1 (32 KB each, rotated, fp16, 128B-swizzled K-major blocks), then a ring of kStages
 // 32 KB slots holding K'_0, V't_0, K'_1, ...
 //
-// Softmax keeps, per row, a reference m (log2 domain) and a row sum l.  m is only raised when a tile's
-// maximum exceeds it by more than kRescaleGap (probabilities stay <= 2^kRescaleGap, inside fp16 range), so
-// after the first tile the probabilities are formed directly against the reference of the earlier tiles,
-// chunk by chunk as the scores arrive; the two threads of a row exchange their half-row maxima through
-// shared memory once per tile, and the rescale of the O accumulator (with a redo of the tile) is rare.
+// Softmax keeps, per row, a reference m (log2 domain) and a row sum l.  m is set from the first tile's row
+// maximum and afterwards only raised when a probability would leave the fp16 range (p = 2^(s - m) > 65504),
+// so the probabilities of a tile are formed directly against the reference of the earlier tiles, chunk by
+// chunk as the scores arrive; the threads of a row exchange one float per tile through shared memory to
+// agree on that, and the rescale of the O accumulator (with a redo of the tile) is rare.
 #include "common.cuh"
 #include "ptx.cuh"
 #include "q_tile.cuh"
@@ -31,11 +31,11 @@ namespace regenvc {
 
 #ifdef REGENVC_TRACE
 // Bring-up instrumentation (never compiled into the shipped library): clock64 stamps of one CTA.
-__device__ long long g_trace[64 * 16];
+__device__ long long g_trace[64 * 32];
 #define TRACE(j, slot)                                                                  \
     do {                                                                                \
         if (blockIdx.x == 3 && blockIdx.y == 0 && (j) >= 16 && (j) < 80)                \
-            g_trace[((j) - 16) * 16 + (slot)] = clock64();                              \
+            g_trace[((j) - 16) * 32 + (slot)] = clock64();                              \
     } while (0)
 #else
 #define TRACE(j, slot) do {} while (0)
@@ -44,19 +44,31 @@ __device__ long long g_trace[64 * 16];
 namespace {
 
 constexpr int kStages = 4;                       // K/V ring slots (32 KB each)
-constexpr int kSoftmaxThreads = 256;
-constexpr int kThreads = kSoftmaxThreads + 128;  // + one warpgroup holding the UMMA and TMA warps
-constexpr int kSoftmaxRegs = 232, kControlRegs = 40;  // 256 * 232 + 128 * 40 <= 64 K registers
-constexpr int kMmaWarp = 8, kTmaWarp = 9;
-constexpr float kRescaleGap = 8.0f;
+#ifndef REGENVC_ROW_SPLIT
+#define REGENVC_ROW_SPLIT 4
+#endif
+constexpr int kSplit = REGENVC_ROW_SPLIT;          // threads sharing one score row (2 or 4)
+constexpr int kColsPerThread = kTile / kSplit;     // key columns of a score tile per thread (64 or 32)
+constexpr int kChunks = kColsPerThread / 32;       // 32-column TMEM loads per thread and tile
+constexpr int kSoftmaxThreads = 128 * kSplit;
+constexpr int kThreads = kSoftmaxThreads + 128;    // + one warpgroup holding the UMMA and TMA warps
+// Register hand-over between the warpgroups (setmaxnreg): what the softmax warps take must fit in what
+// the CTA got at launch (kLaunchRegs per thread, checked against the compiled kernel on the host)
+// minus what the control warpgroup keeps; an over-ask would block the last softmax warpgroup forever.
+constexpr int kLaunchRegs = (65536 / kThreads) / 8 * 8;   // 168 for 384 threads, 96 for 640
+constexpr int kControlRegs = 40;
+constexpr int kSoftmaxRegs = ((kLaunchRegs * kThreads - kControlRegs * 128) / kSoftmaxThreads) / 8 * 8;  // 232 / 104
+static_assert(kSoftmaxRegs * kSoftmaxThreads + kControlRegs * 128 <= kLaunchRegs * kThreads, "register budget");
+static_assert(kSoftmaxRegs >= kLaunchRegs && kSoftmaxRegs <= 255, "setmaxnreg.inc must not shrink");
+constexpr int kMmaWarp = kSoftmaxThreads / 32, kTmaWarp = kMmaWarp + 1;
 #ifndef REGENVC_POLY_MASK
 #define REGENVC_POLY_MASK 0x52
 #endif
 // bit i set: pair i of every eight probability pairs takes the polynomial 2^x instead of the MUFU
 constexpr uint32_t kPolyMask = REGENVC_POLY_MASK;
 constexpr uint32_t kIdesc = umma_idesc_f16_f32acc(128, 128);
-constexpr uint32_t kSmemBytes = (2 + kStages) * kTileBytes + 1024 /*align*/ + 256 /*barriers*/ + 6144 /*row exchange*/;
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
+constexpr uint32_t kSmemBytes = (2 + kStages) * kTileBytes + 1024 /*align*/ + 256 /*barriers*/ + 16384 /*row exchange*/;
+constexpr uint64_t kWaitLimitNs = 500000000ull;   // 0.5 s per wait
 
 struct Barriers {
     uint64_t kv_full[kStages];
@@ -72,8 +84,9 @@ static_assert(sizeof(Barriers) <= 256, "barrier block too large");
 
 // Values the two threads of a row hand each other: [parity][tile][half][row].
 struct RowExchange {
-    float v[2][2][2][kTile];
-    float l[2][2][kTile];  // row sums at the end: [tile][half][row]
+    float v[2][2][kTile][kSplit];  // partial tile sums: [parity][tile][row][part]
+    float m[2][kTile][kSplit];     // partial tile maxima (redo path): [tile][row][part]
+    float l[2][kTile][kSplit];     // row sums at the end: [tile][row][part]
 };
 
 // 2^x for a packed pair on the FMA/ALU pipes: x = n + f with n = round(x), f in [-0.5, 0.5];
@@ -86,7 +99,7 @@ __device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
     const float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
     const uint64_t r2 = add2(x2, pack2(kMagic, kMagic));
     const uint64_t n2 = add2(r2, pack2(-kMagic, -kMagic));
-    const uint64_t f2 = add2(x2, mul2(n2, pack2(-1.0f, -1.0f)));
+    const uint64_t f2 = fma2(n2, pack2(-1.0f, -1.0f), x2);
     uint64_t q2 = fma2(f2, pack2(0.0551716685f, 0.0551716685f), pack2(0.242611125f, 0.242611125f));
     q2 = fma2(q2, f2, pack2(0.693260968f, 0.693260968f));
     q2 = fma2(q2, f2, pack2(0.999928057f, 0.999928057f));
@@ -98,9 +111,13 @@ __device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
     return pack2(q0, q1);
 }
 
-// Named barrier over the eight softmax warps (barrier 0 is __syncthreads).
+// Named barrier over all softmax warps (barrier 0 is __syncthreads).
 __device__ __forceinline__ void softmax_barrier() {
     asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
+}
+// Named barrier over the kSplit warps that share the 32 rows of lane group g (barriers 2..5).
+__device__ __forceinline__ void row_group_barrier(int g) {
+    asm volatile("bar.sync %0, %1;" ::"r"(2 + g), "n"(32 * kSplit) : "memory");
 }
 
 // 32 scores of one row -> 16 packed fp16 probability pairs p = 2^(s * scale - m_ref).  The FMA is done on
@@ -125,7 +142,7 @@ __device__ __forceinline__ void exp_chunk(const uint32_t* s, uint64_t scale2, ui
         else sum_a = add2(sum_a, p2);
         float p0, p1;
         unpack2(p2, p0, p1);
-        pr[c] = pack_f16x2(p0, p1);
+        pr[c] = pack_f16x2_sat(p0, p1);
     }
 }
 
@@ -144,8 +161,10 @@ __device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint3
 #pragma unroll
     for (int kk = 0; kk < 8; ++kk) {
         const uint64_t off = (kk >> 2) * (kBlockBytes >> 4) + (kk & 3) * 2;
-        // P: keys 0..63 at columns [0,32), keys 64..127 at columns [64,96) of the score tile
-        umma_ts(d_tmem, p_tmem + (kk >> 2) * 64 + (kk & 3) * 8, b0 + off, kIdesc, accumulate || kk > 0);
+        // P of keys [c, c + kColsPerThread) sits in the first half of score columns [c, c + kColsPerThread)
+        constexpr int kGroups = kColsPerThread / 16;  // 16-key MMA steps per column group
+        umma_ts(d_tmem, p_tmem + (kk / kGroups) * kColsPerThread + (kk % kGroups) * 8, b0 + off, kIdesc,
+                accumulate || kk > 0);
     }
 }
 
@@ -178,7 +197,8 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             mbar_init(smem_u32(&bar->p_full[t]), kSoftmaxThreads);
             mbar_init(smem_u32(&bar->o_full[t]), 1);
         }
-        bar->abort_flag = 0;
+        // a sticky error from an earlier kernel makes this CTA skip its work (every bounded wait falls through)
+        bar->abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0) ? 1 : 0;
         fence_mbar_init();
     }
     if (warp == kMmaWarp) {
@@ -264,7 +284,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     } else {
         // ------------------------------------------------------------ softmax groups
         setmaxnreg_inc<kSoftmaxRegs>();
-        const int half = warp >> 2;                      // which 64 key columns of a score row
+        const int part = warp >> 2;                      // which kColsPerThread key columns of a score row
         const int row = (warp & 3) * 32 + lane;          // row in the tile == TMEM lane
         const int n_active = tile1_active ? 2 : 1;
         for (int t = 0; t < n_active; ++t) {
@@ -282,36 +302,34 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
                 if (t >= n_active) continue;
-                const uint32_t t_S = lane_base + t * 128 + half * 64, t_O = lane_base + 256 + t * 128 + half * 64;
+                const uint32_t t_S = lane_base + t * 128 + part * kColsPerThread;
+                const uint32_t t_O = lane_base + 256 + t * 128 + part * kColsPerThread;
                 if (tid == 0) TRACE(j, t * 6 + 0);
                 if (ok) ok = mbar_wait(smem_u32(&bar->s_full[t]), j & 1, ctl);
                 ok = __all_sync(0xffffffffu, ok);  // keep the warp-wide TMEM instructions below convergent
                 tc_fence_after();
                 if (tid == 0) TRACE(j, t * 6 + 1);
-                uint32_t sr[64];
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-                const int valid = ((j == n_tiles - 1) ? p.n_kv - j * kTile : kTile) - half * 64;  // own columns >= valid are padding
+                // From the second tile on, the probabilities of each 32-column chunk are formed as soon as it
+                // arrives, against the reference m_ref of the earlier tiles; no maximum is taken.  Probabilities
+                // saturate at 65504 when rounded to fp16, and a saturated one makes the fp32 sum of its part reach
+                // 65504, which the threads of the row detect by exchanging their sums; only then (and on the first
+                // tile) the row maximum is taken, the reference raised, O rescaled and the tile redone.
+                uint32_t sr[kColsPerThread];
+                // own columns >= valid are padding
+                const int valid = ((j == n_tiles - 1) ? p.n_kv - j * kTile : kTile) - part * kColsPerThread;
                 uint64_t negm2 = pack2(-m_ref[t], -m_ref[t]);
                 uint64_t sum_a = 0, sum_b = 0;  // packed partial row sums
                 const bool stream = j > 0;
                 if (ok) {
                     tmem_ld32(t_S, sr);
 #pragma unroll
-                    for (int cb = 0; cb < 2; ++cb) {
+                    for (int cb = 0; cb < kChunks; ++cb) {
                         tmem_wait_ld();
-                        if (cb == 0) tmem_ld32(t_S + 32, sr + 32);
-                        if (valid < 64) {
+                        if (cb + 1 < kChunks) tmem_ld32(t_S + 32 * (cb + 1), sr + 32 * (cb + 1));
+                        if (valid < kColsPerThread) {
 #pragma unroll
                             for (int c = 0; c < 32; ++c)
                                 if (cb * 32 + c >= valid) sr[cb * 32 + c] = 0xff800000u;  // -inf
-                        }
-#pragma unroll
-                        for (int c = 0; c < 32; c += 8) {
-                            const uint32_t* x = sr + cb * 32 + c;
-                            mx0 = max3(mx0, __uint_as_float(x[0]), __uint_as_float(x[1]));
-                            mx1 = max3(mx1, __uint_as_float(x[2]), __uint_as_float(x[3]));
-                            mx2 = max3(mx2, __uint_as_float(x[4]), __uint_as_float(x[5]));
-                            mx3 = max3(mx3, __uint_as_float(x[6]), __uint_as_float(x[7]));
                         }
                         if (stream) {
                             uint32_t pr[16];
@@ -320,26 +338,48 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                         }
                     }
                 }
-                // the two threads of a row exchange their half-row maxima
-                const float mx_half = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                xch->v[j & 1][t][half][row] = mx_half;
-                softmax_barrier();
-                const float m_tile = fmaxf(mx_half, xch->v[j & 1][t][half ^ 1][row]) * scale;
+                float part_sum;
+                {
+                    float s0, s1;
+                    unpack2(add2(sum_a, sum_b), s0, s1);
+                    part_sum = s0 + s1;
+                }
+                xch->v[j & 1][t][row][part] = part_sum;
+                row_group_barrier(warp & 3);
+                bool redo = !stream || !(part_sum < 65504.0f);
+#pragma unroll
+                for (int o = 1; o < kSplit; ++o) redo |= !(xch->v[j & 1][t][row][(part + o) % kSplit] < 65504.0f);
                 if (tid == 0) TRACE(j, t * 6 + 2);
-                const bool raise = m_tile > m_ref[t] + kRescaleGap;  // always true on the first tile
-                const bool any_raise = __any_sync(0xffffffffu, raise);
-                if (ok && any_raise) {
-                    // some row of this warp moves its reference (the partner warp sees the same rows and takes
-                    // the same branch): rescale this thread's half of the O row and its row sum, then (re)compute
-                    // the probabilities of the tile against the new reference
+                const bool any_redo = __any_sync(0xffffffffu, redo);
+                if (any_redo) {
+                    // Rare after the first tile.  The warps sharing these rows see the same flags and take the
+                    // same branch: row maximum, new reference for the flagged rows, rescale of this thread's part
+                    // of the O row and of its row sum, then the probabilities of the tile against the reference.
+                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                    for (int c = 0; c < kColsPerThread; c += 8) {
+                        mx0 = max3(mx0, __uint_as_float(sr[c + 0]), __uint_as_float(sr[c + 1]));
+                        mx1 = max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
+                        mx2 = max3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
+                        mx3 = max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
+                    }
+                    const float mx_part = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                    xch->m[t][row][part] = mx_part;
+                    row_group_barrier(warp & 3);
+                    float mx_row = mx_part;
+#pragma unroll
+                    for (int o = 1; o < kSplit; ++o) mx_row = fmaxf(mx_row, xch->m[t][row][(part + o) % kSplit]);
+                    row_group_barrier(warp & 3);  // everyone has read xch->m before a later redo overwrites it
+                    const float m_tile = mx_row * scale;
                     if (j > 0) {
-                        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar->o_full[t]), (j - 1) & 1, ctl));
+                        if (ok) ok = mbar_wait(smem_u32(&bar->o_full[t]), (j - 1) & 1, ctl);
+                        ok = __all_sync(0xffffffffu, ok);
                         tc_fence_after();
-                        const float alpha = raise ? ex2_approx(m_ref[t] - m_tile) : 1.0f;
+                        const float alpha = redo ? ex2_approx(m_ref[t] - m_tile) : 1.0f;
                         l_run[t] *= alpha;
                         if (ok) {
 #pragma unroll 1
-                            for (int cb = 0; cb < 2; ++cb) {
+                            for (int cb = 0; cb < kChunks; ++cb) {
                                 uint32_t o[32];
                                 tmem_ld32(t_O + cb * 32, o);
                                 tmem_wait_ld();
@@ -349,13 +389,13 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                             }
                         }
                     }
-                    if (raise) m_ref[t] = m_tile;
+                    if (redo) m_ref[t] = m_tile;
                     negm2 = pack2(-m_ref[t], -m_ref[t]);
                     sum_a = 0;
                     sum_b = 0;
                     if (ok) {
 #pragma unroll
-                        for (int cb = 0; cb < 2; ++cb) {
+                        for (int cb = 0; cb < kChunks; ++cb) {
                             uint32_t pr[16];
                             exp_chunk<kPolyMask>(sr + cb * 32, scale2, negm2, pr, sum_a, sum_b);
                             tmem_st16(t_S + cb * 16, pr);
@@ -373,25 +413,29 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             }
         }
 
-        // epilogue: O / l -> bf16 -> out; each thread owns 64 of the 128 output columns of its row
+        // epilogue: O / l -> bf16 -> out; each thread owns kColsPerThread of the 128 output columns of its row
         for (int t = 0; t < n_active; ++t) {
-            xch->l[t][half][row] = l_run[t];
+            xch->l[t][row][part] = l_run[t];
             softmax_barrier();
-            const float inv_l = 1.0f / (l_run[t] + xch->l[t][half ^ 1][row]);
+            float l_row = 0.f;
+#pragma unroll
+            for (int o = 0; o < kSplit; ++o) l_row += xch->l[t][row][o];
+            const float inv_l = 1.0f / l_row;
             if (ok) ok = mbar_wait(smem_u32(&bar->o_full[t]), (n_tiles - 1) & 1, ctl);
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
             const int n = q0 + t * kTile + row;
-            const uint32_t t_O = lane_base + 256 + t * 128 + half * 64;
+            const uint32_t t_O = lane_base + 256 + t * 128 + part * kColsPerThread;
 #pragma unroll 1
-            for (int cb = 0; cb < 2; ++cb) {
+            for (int cb = 0; cb < kChunks; ++cb) {
                 uint32_t o[32];
                 if (ok) {
                     tmem_ld32(t_O + cb * 32, o);
                     tmem_wait_ld();
                 }
                 if (ok && n < p.n_q) {
-                    uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)n * p.h + head) * kHeadDim + half * 64 + cb * 32);
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)n * p.h + head) * kHeadDim +
+                                                          part * kColsPerThread + cb * 32);
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint4 w;
@@ -429,6 +473,11 @@ extern "C" int regenvc_debug_read_trace(long long* out) {
 #endif
 
 cudaError_t configure_attn_pipelined() {
+    cudaFuncAttributes attr;
+    cudaError_t e = cudaFuncGetAttributes(&attr, attn_pipelined_kernel);
+    if (e != cudaSuccess) return e;
+    // the register hand-over above assumes the kernel was compiled to exactly kLaunchRegs registers per thread
+    if (attr.numRegs != kLaunchRegs) return cudaErrorInvalidConfiguration;
     return cudaFuncSetAttribute(attn_pipelined_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
 }
 
