@@ -102,8 +102,11 @@ int regenvc_cross_attn_forward_host(const void* q, const void* k, const void* v,
  *   K' : fp16 [n_heads][n_kv_pad][128]   rotated (self) or converted (cross) keys
  *   V't: fp16 [n_heads][128][n_kv_pad]   values, transposed so that keys are contiguous
  * with n_kv_pad = n_kv rounded up to a multiple of 128 (padding is zero),
- * K' first, V't directly after it.  regenvc_workspace_bytes() returns the
- * size this needs (0 for invalid arguments).  By default the library keeps
+ * K' first, V't directly after it, followed by a fixed 21,299,200-byte area
+ * for the partial results of query tiles whose key range is cut into pieces
+ * (fp32 accumulators, references and row sums that a merge kernel combines).
+ * regenvc_workspace_bytes() returns the total this needs (0 for invalid
+ * arguments).  By default the library keeps
  * one workspace per device and host thread and grows it on demand with
  * cudaMalloc (which synchronises: do a warm-up call before capturing a CUDA
  * graph).  regenvc_set_workspace() makes the calling host thread use a

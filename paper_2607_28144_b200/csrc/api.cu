@@ -73,6 +73,14 @@ bool serial_kernel_requested() {
     return serial;
 }
 
+bool split_disabled() {
+    static const bool off = [] {
+        const char* e = std::getenv("REGENVC_SPLIT_KV");
+        return e && std::strcmp(e, "0") == 0;
+    }();
+    return off;
+}
+
 bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
     const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
     return a0 < b0 + nb && b0 < a0 + na;
@@ -184,10 +192,11 @@ int make_tmap(CUtensorMap* m, void* base, uint64_t inner, uint64_t outer, uint64
     return REGENVC_OK;
 }
 
-size_t workspace_need(long long n_kv, int n_heads) {
+size_t operand_bytes(long long n_kv, int n_heads) {
     const size_t kv_pad = (size_t)((n_kv + kTile - 1) / kTile * kTile);
     return 2 * (size_t)n_heads * kv_pad * kHeadDim * sizeof(__half);
 }
+size_t workspace_need(long long n_kv, int n_heads) { return operand_bytes(n_kv, n_heads) + kSplitScratchBytes; }
 
 // Enqueues the two kernels.  Arguments are already validated; pointers are device pointers.
 int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int n_kv, int n_heads, bool rope, int T,
@@ -254,11 +263,48 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)kHeadDim));
     ap.status = st->status;
     ap.sm_count = st->sm_count;
-    if (serial_kernel_requested())
+    // Work decomposition: one CTA per (head, 256 query rows).  The items of the last, incomplete wave are cut
+    // along the key axis into split_k pieces each so that the pieces fill the SMs; a merge kernel combines them.
+    const int n_tiles = kv_pad / kTile;
+    ap.pairs_per_head = (n_q + 2 * kTile - 1) / (2 * kTile);
+    const int n_items = ap.pairs_per_head * n_heads;
+    ap.n_full_items = n_items;
+    ap.split_k = 1;
+    ap.tiles_per_piece = n_tiles;
+    ap.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + operand_bytes(n_kv, n_heads));
+    ap.part_ml = reinterpret_cast<float2*>(ap.part_o + (size_t)kMaxPieceCtas * 2 * kTile * kHeadDim);
+    const int rem = n_items % st->sm_count;
+    if (rem > 0 && st->sm_count <= kMaxPieceCtas && !split_disabled()) {
+        int k = st->sm_count / rem;
+        if (k > 8) k = 8;
+        if (k > n_tiles / 4) k = n_tiles / 4;
+        if (k >= 2) {
+            ap.tiles_per_piece = (n_tiles + k - 1) / k;
+            ap.split_k = (n_tiles + ap.tiles_per_piece - 1) / ap.tiles_per_piece;  // no empty piece
+            ap.n_full_items = n_items - rem;
+        }
+    }
+    if (serial_kernel_requested()) {
         CUDA_TRY(launch_attn_serial(tmap_k, tmap_v, ap, stream));
-    else
-        CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, ap, stream));
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return REGENVC_OK;
+    }
+    CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, ap, stream));
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (ap.split_k > 1) {
+        MergeParams mp;
+        mp.part_o = ap.part_o;
+        mp.part_ml = ap.part_ml;
+        mp.out = ap.out;
+        mp.n_q = n_q;
+        mp.h = n_heads;
+        mp.pairs_per_head = ap.pairs_per_head;
+        mp.n_full_items = ap.n_full_items;
+        mp.split_k = ap.split_k;
+        mp.n_split_items = n_items - ap.n_full_items;
+        CUDA_TRY(launch_merge_partials(mp, stream));
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
     return REGENVC_OK;
 }
 

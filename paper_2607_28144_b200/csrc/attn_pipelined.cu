@@ -34,7 +34,7 @@ namespace regenvc {
 __device__ long long g_trace[64 * 32];
 #define TRACE(j, slot)                                                                  \
     do {                                                                                \
-        if (blockIdx.x == 3 && blockIdx.y == 0 && (j) >= 16 && (j) < 80)                \
+        if (blockIdx.x == 3 && (j) >= 16 && (j) < 80)                \
             g_trace[((j) - 16) * 32 + (slot)] = clock64();                              \
     } while (0)
 #else
@@ -181,10 +181,19 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     RowExchange* xch = reinterpret_cast<RowExchange*>(base + (2 + kStages) * kTileBytes + 256);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int head = blockIdx.y;
-    const int q0 = blockIdx.x * 2 * kTile;
+    // work item and key-tile range of this CTA
+    const int n_tiles_total = p.n_kv_pad / kTile;
+    int item = blockIdx.x, kv_tile0 = 0, n_tiles = n_tiles_total;
+    const bool partial = static_cast<int>(blockIdx.x) >= p.n_full_items;
+    const int piece_cta = static_cast<int>(blockIdx.x) - p.n_full_items;
+    if (partial) {
+        item = p.n_full_items + piece_cta / p.split_k;
+        kv_tile0 = (piece_cta % p.split_k) * p.tiles_per_piece;
+        n_tiles = min(p.tiles_per_piece, n_tiles_total - kv_tile0);
+    }
+    const int head = item / p.pairs_per_head;
+    const int q0 = (item % p.pairs_per_head) * 2 * kTile;
     const bool tile1_active = q0 + kTile < p.n_q;
-    const int n_tiles = p.n_kv_pad / kTile;
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -227,7 +236,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 if (round > 0 && !mbar_wait(smem_u32(&bar->kv_empty[slot]), (round - 1) & 1, ctl)) break;
                 const uint32_t full = smem_u32(&bar->kv_full[slot]);
                 const uint32_t dst = smem_u32(sKV + slot * kTileBytes);
-                const int kv0 = (i >> 1) * kTile;
+                const int kv0 = (kv_tile0 + (i >> 1)) * kTile;
                 mbar_expect_tx(full, kTileBytes);
                 if ((i & 1) == 0) {
                     tma_load_2d(dst, &tmap_k, 0, head * p.n_kv_pad + kv0, full);
@@ -316,7 +325,8 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 // tile) the row maximum is taken, the reference raised, O rescaled and the tile redone.
                 uint32_t sr[kColsPerThread];
                 // own columns >= valid are padding
-                const int valid = ((j == n_tiles - 1) ? p.n_kv - j * kTile : kTile) - part * kColsPerThread;
+                const int valid = ((kv_tile0 + j == n_tiles_total - 1) ? p.n_kv - (kv_tile0 + j) * kTile : kTile) -
+                                  part * kColsPerThread;
                 uint64_t negm2 = pack2(-m_ref[t], -m_ref[t]);
                 uint64_t sum_a = 0, sum_b = 0;  // packed partial row sums
                 const bool stream = j > 0;
@@ -426,6 +436,8 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             tc_fence_after();
             const int n = q0 + t * kTile + row;
             const uint32_t t_O = lane_base + 256 + t * 128 + part * kColsPerThread;
+            if (partial && part == 0)
+                p.part_ml[(size_t)piece_cta * 2 * kTile + t * kTile + row] = make_float2(m_ref[t], l_row);
 #pragma unroll 1
             for (int cb = 0; cb < kChunks; ++cb) {
                 uint32_t o[32];
@@ -433,7 +445,13 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     tmem_ld32(t_O + cb * 32, o);
                     tmem_wait_ld();
                 }
-                if (ok && n < p.n_q) {
+                if (ok && partial) {
+                    // unnormalised fp32 row part for the merge kernel
+                    uint4* dst = reinterpret_cast<uint4*>(p.part_o + ((size_t)piece_cta * 2 * kTile + t * kTile + row) * kHeadDim +
+                                                          part * kColsPerThread + cb * 32);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) dst[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                } else if (ok && n < p.n_q) {
                     uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)n * p.h + head) * kHeadDim +
                                                           part * kColsPerThread + cb * 32);
 #pragma unroll
@@ -483,7 +501,8 @@ cudaError_t configure_attn_pipelined() {
 
 cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const AttnParams& p,
                                   cudaStream_t stream) {
-    dim3 grid((p.n_q + 2 * kTile - 1) / (2 * kTile), p.h);
+    const int n_items = p.pairs_per_head * p.h;
+    dim3 grid(p.n_full_items + (n_items - p.n_full_items) * p.split_k);
     attn_pipelined_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmap_k, tmap_v, p);
     return cudaGetLastError();
 }

@@ -47,9 +47,34 @@ struct AttnParams {
     float scale_log2;         // log2(e) / sqrt(head_dim)
     int* status;
     int sm_count;
+    // Work decomposition of the pipelined kernel.  A work item is one head and 256 query rows; items are
+    // numbered head-major.  The first n_full_items CTAs each run one item over all keys.  Each of the remaining
+    // items is cut into split_k pieces of tiles_per_piece key tiles, one CTA per piece, which leave
+    // unnormalised partial results in part_o / part_ml for the merge kernel.
+    int pairs_per_head;       // items per head = ceil(n_q / 256)
+    int n_full_items;
+    int split_k;              // >= 1
+    int tiles_per_piece;
+    float* part_o;            // [piece CTA][256 rows][128] fp32, sum_m p_m v_m against the piece's reference
+    float2* part_ml;          // [piece CTA][256 rows] (reference m in log2 units, row sum l)
+};
+
+struct MergeParams {
+    const float* part_o;
+    const float2* part_ml;
+    __nv_bfloat16* out;       // [n_q, h, 128]
+    int n_q, h;
+    int pairs_per_head, n_full_items, split_k, n_split_items;
 };
 
 // Launchers (each returns the launch error, enqueues on `stream`).
 cudaError_t launch_prep_kv(const PrepParams& p, cudaStream_t stream);
+cudaError_t launch_merge_partials(const MergeParams& p, cudaStream_t stream);
+
+// Bytes of the partial-result scratch that follows K' and V't in the workspace: room for up to
+// kMaxPieceCtas piece CTAs (never more than one wave of SMs is cut into pieces).
+constexpr int kMaxPieceCtas = 160;
+constexpr size_t kPieceBytes = 2 * kTile * kHeadDim * sizeof(float) + 2 * kTile * sizeof(float2);
+constexpr size_t kSplitScratchBytes = kMaxPieceCtas * kPieceBytes;
 
 }  // namespace regenvc

@@ -40,10 +40,12 @@ def test_status_strings_and_version(L):
 
 
 def test_workspace_bytes():
-    # K' and V't, fp16, key count padded to 128
-    assert binding.regenvc_workspace_bytes(10920, 12) == 2 * 12 * 11008 * 128 * 2
-    assert binding.regenvc_workspace_bytes(128, 2) == 2 * 2 * 128 * 128 * 2
-    assert binding.regenvc_workspace_bytes(1, 1) == 2 * 128 * 128 * 2
+    # K' and V't, fp16, key count padded to 128, plus the fixed split-key scratch
+    scratch = 160 * (256 * 128 * 4 + 256 * 8)
+    assert scratch == 21_299_200
+    assert binding.regenvc_workspace_bytes(10920, 12) == 2 * 12 * 11008 * 128 * 2 + scratch
+    assert binding.regenvc_workspace_bytes(128, 2) == 2 * 2 * 128 * 128 * 2 + scratch
+    assert binding.regenvc_workspace_bytes(1, 1) == 2 * 128 * 128 * 2 + scratch
     assert binding.regenvc_workspace_bytes(0, 1) == 0
     assert binding.regenvc_workspace_bytes(5, 1, 64) == 0
 

@@ -35,14 +35,14 @@ def test_workspace_holds_rotated_keys_and_transposed_values():
     rng = np.random.default_rng(5)
     q, k, v = _rand(rng, N, h), _rand(rng, N, h), _rand(rng, N, h)
     nbytes = binding.regenvc_workspace_bytes(N, h)
-    assert nbytes == 2 * h * n_pad * D * 2
+    assert nbytes == 2 * h * n_pad * D * 2 + 21_299_200
     ws = torch.full((nbytes,), 0xFF, dtype=torch.uint8, device="cuda:0")
     binding.regenvc_set_workspace(ws)
     try:
         run_gpu_self(q, k, v, T, H, W)
     finally:
         binding.regenvc_set_workspace(None)
-    halves = ws.view(torch.float16).cpu()
+    halves = ws[: 2 * h * n_pad * D * 2].view(torch.float16).cpu()
     kp = halves[: h * n_pad * D].view(h, n_pad, D).double().numpy()
     vt = halves[h * n_pad * D:].view(h, D, n_pad).double().numpy()
     for a in range(h):
@@ -72,6 +72,22 @@ def test_self_attention_window_256x256():
     for a in range(w.n_heads):  # per head, to localise a bad head
         assert errors(gpu[:, a], ref[:, a], float(v.float().abs().max()))["mre"] <= 2e-3
     print("window_256x256", e)
+
+
+@pytest.mark.parametrize("grid,h", [((7, 16, 16), 2), ((1, 25, 44), 3), ((2, 37, 29), 1), ((1, 40, 64), 5)])
+def test_self_attention_with_split_key_pieces(grid, h):
+    """Few work items and many key tiles: the library cuts the key range of every item into pieces (the
+    incomplete-last-wave path) and merges the partial results; uneven pieces and a ragged last tile included."""
+    T, H, W = grid
+    _self_case(T, H, W, h, seed=4000 + T * H * W + h)
+
+
+def test_cross_attention_with_split_key_pieces():
+    rng = np.random.default_rng(4100)
+    q, k, v = _rand(rng, 300, 2), _rand(rng, 1500, 2), _rand(rng, 1500, 2)
+    gpu = f64(run_gpu_cross(q, k, v))
+    ref = oracle.cross_attention(synth.bits(q), synth.bits(k), synth.bits(v))
+    assert_parity(gpu, ref, float(v.float().abs().max()), "cross 300x1500 split")
 
 
 def test_tiny_workload_against_brute_force_too():
