@@ -17,7 +17,6 @@ namespace regenvc {
 cudaError_t configure_attn_serial();
 cudaError_t launch_attn_serial(const CUtensorMap&, const CUtensorMap&, const AttnParams&, cudaStream_t);
 cudaError_t configure_attn_pipelined();
-cudaError_t launch_attn_pipelined(const CUtensorMap&, const CUtensorMap&, const AttnParams&, cudaStream_t);
 }  // namespace regenvc
 
 namespace {
@@ -177,12 +176,13 @@ int rope_table(DeviceState& st, int T, int H, int W, float theta, const float2**
     return REGENVC_OK;
 }
 
-int make_tmap(CUtensorMap* m, void* base, uint64_t inner, uint64_t outer, uint64_t row_bytes) {
+int make_tmap(CUtensorMap* m, void* base, uint64_t inner, uint64_t outer, uint64_t row_bytes,
+              CUtensorMapDataType type = CU_TENSOR_MAP_DATA_TYPE_FLOAT16) {
     const cuuint64_t gdim[2] = {inner, outer};
     const cuuint64_t gstride[1] = {row_bytes};
     const cuuint32_t box[2] = {64, 128};
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, gdim, gstride, box, estr,
+    CUresult r = g_encode(m, type, 2, base, gdim, gstride, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -289,7 +289,12 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
         g_launches.fetch_add(1, std::memory_order_relaxed);
         return REGENVC_OK;
     }
-    CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, ap, stream));
+    // out seen as [n_q rows][n_heads * 128 columns] bf16 for the tiled stores of finished query tiles
+    CUtensorMap tmap_out;
+    rc = make_tmap(&tmap_out, out, (uint64_t)n_heads * kHeadDim, (uint64_t)n_q,
+                   (uint64_t)n_heads * kHeadDim * sizeof(__nv_bfloat16), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
+    if (rc != REGENVC_OK) return rc;
+    CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, ap, stream));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (ap.split_k > 1) {
         MergeParams mp;

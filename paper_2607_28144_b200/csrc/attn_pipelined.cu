@@ -37,8 +37,13 @@ __device__ long long g_trace[64 * 32];
         if (blockIdx.x == 3 && (j) >= 16 && (j) < 80)                \
             g_trace[((j) - 16) * 32 + (slot)] = clock64();                              \
     } while (0)
+#define TRACE_CTA(slot)                                                                 \
+    do {                                                                                \
+        if (blockIdx.x == 3) g_trace[63 * 32 + (slot)] = clock64();                     \
+    } while (0)
 #else
 #define TRACE(j, slot) do {} while (0)
+#define TRACE_CTA(slot) do {} while (0)
 #endif
 
 namespace {
@@ -172,7 +177,7 @@ __device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint3
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
-                      const AttnParams p) {
+                      const __grid_constant__ CUtensorMap tmap_out, const AttnParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = base;                       // 2 tiles
@@ -195,6 +200,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     const int q0 = (item % p.pairs_per_head) * 2 * kTile;
     const bool tile1_active = q0 + kTile < p.n_q;
 
+    if (tid == 0) TRACE_CTA(0);
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_u32(&bar->kv_full[s]), 1);
@@ -217,11 +223,13 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     if (warp == kTmaWarp && elect_one()) {
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
+        tma_prefetch_desc(&tmap_out);
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
 
+    if (tid == 0) TRACE_CTA(1);
     const uint32_t tmem_base = bar->tmem_base;
     const WaitCtl ctl{&bar->abort_flag, p.status, kStatusTimeout, kWaitLimitNs};
 
@@ -296,11 +304,11 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         const int part = warp >> 2;                      // which kColsPerThread key columns of a score row
         const int row = (warp & 3) * 32 + lane;          // row in the tile == TMEM lane
         const int n_active = tile1_active ? 2 : 1;
-        for (int t = 0; t < n_active; ++t) {
-            load_rotate_q_tile(p, head, q0 + t * kTile, sQ + t * kTileBytes, tid, kSoftmaxThreads);
-            fence_proxy_async_smem();
-            mbar_arrive(smem_u32(&bar->q_full[t]));
-        }
+        if (tile1_active) load_rotate_q_tiles<kSoftmaxThreads, 2>(p, head, q0, sQ, tid);
+        else load_rotate_q_tiles<kSoftmaxThreads, 1>(p, head, q0, sQ, tid);
+        fence_proxy_async_smem();
+        for (int t = 0; t < n_active; ++t) mbar_arrive(smem_u32(&bar->q_full[t]));
+        if (tid == 0) TRACE_CTA(2);
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         const float scale = p.scale_log2;
         const uint64_t scale2 = pack2(scale, scale);
@@ -318,6 +326,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 ok = __all_sync(0xffffffffu, ok);  // keep the warp-wide TMEM instructions below convergent
                 tc_fence_after();
                 if (tid == 0) TRACE(j, t * 6 + 1);
+                if (tid == 0 && j == 0 && t == 0) TRACE_CTA(3);
                 // From the second tile on, the probabilities of each 32-column chunk are formed as soon as it
                 // arrives, against the reference m_ref of the earlier tiles; no maximum is taken.  Probabilities
                 // saturate at 65504 when rounded to fp16, and a saturated one makes the fp32 sum of its part reach
@@ -420,8 +429,10 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bar->p_full[t]));
                 if (tid == 0) TRACE(j, t * 6 + 4);
+                if (tid == 0 && j == 0 && t == 0) TRACE_CTA(4);
             }
         }
+        if (tid == 0) TRACE_CTA(5);
 
         // epilogue: O / l -> bf16 -> out; each thread owns kColsPerThread of the 128 output columns of its row
         for (int t = 0; t < n_active; ++t) {
@@ -434,6 +445,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             if (ok) ok = mbar_wait(smem_u32(&bar->o_full[t]), (n_tiles - 1) & 1, ctl);
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
+            if (tid == 0) TRACE_CTA(6 + t);
             const int n = q0 + t * kTile + row;
             const uint32_t t_O = lane_base + 256 + t * 128 + part * kColsPerThread;
             if (partial && part == 0)
@@ -451,9 +463,10 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                                                           part * kColsPerThread + cb * 32);
 #pragma unroll
                     for (int c = 0; c < 8; ++c) dst[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
-                } else if (ok && n < p.n_q) {
-                    uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)n * p.h + head) * kHeadDim +
-                                                          part * kColsPerThread + cb * 32);
+                } else if (ok) {
+                    // normalised bf16 row part into the (now idle) query tile buffer, in the swizzled layout of a
+                    // TMA box {64 columns, 128 rows}; one tiled store per 64-column block writes the tile out
+                    uint8_t* stage = sQ + t * kTileBytes;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint4 w;
@@ -461,14 +474,29 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                         w.y = pack_bf16x2(__uint_as_float(o[8 * c + 2]) * inv_l, __uint_as_float(o[8 * c + 3]) * inv_l);
                         w.z = pack_bf16x2(__uint_as_float(o[8 * c + 4]) * inv_l, __uint_as_float(o[8 * c + 5]) * inv_l);
                         w.w = pack_bf16x2(__uint_as_float(o[8 * c + 6]) * inv_l, __uint_as_float(o[8 * c + 7]) * inv_l);
-                        dst[c] = w;
+                        const int col = part * kColsPerThread + cb * 32 + c * 8;  // first of 8 output columns
+                        *reinterpret_cast<uint4*>(stage + (col >> 6) * kBlockBytes + sw128_offset(row, (col >> 3) & 7)) = w;
                     }
                 }
             }
+            if (!partial) {
+                fence_proxy_async_smem();
+                softmax_barrier();
+                if (tid == 0 && ok) {
+                    const uint32_t src = smem_u32(sQ + t * kTileBytes);
+                    tma_store_2d(&tmap_out, head * kHeadDim, q0 + t * kTile, src);
+                    tma_store_2d(&tmap_out, head * kHeadDim + 64, q0 + t * kTile, src + kBlockBytes);
+                    tma_store_commit();
+                }
+            }
         }
+        // the tiled stores read shared memory asynchronously: they must be done before the CTA may exit
+        if (tid == 0 && !partial) tma_store_wait_read();
+        __syncwarp();
     }
 
     // ---------------------------------------------------------------- tear-down
+    if (tid == 0) TRACE_CTA(8);
     __syncwarp();  // lanes that left a single-lane role loop rejoin before the warp-wide instructions below
     tc_fence_before();
     __syncthreads();
@@ -481,6 +509,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         }
         __syncwarp();
         tmem_dealloc(tmem_base, 512);
+        if (lane == 0) TRACE_CTA(9);
     }
 }
 
@@ -499,11 +528,11 @@ cudaError_t configure_attn_pipelined() {
     return cudaFuncSetAttribute(attn_pipelined_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
 }
 
-cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const AttnParams& p,
-                                  cudaStream_t stream) {
+cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
+                                  const AttnParams& p, cudaStream_t stream) {
     const int n_items = p.pairs_per_head * p.h;
     dim3 grid(p.n_full_items + (n_items - p.n_full_items) * p.split_k);
-    attn_pipelined_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmap_k, tmap_v, p);
+    attn_pipelined_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmap_k, tmap_v, tmap_out, p);
     return cudaGetLastError();
 }
 

@@ -52,7 +52,7 @@ attn_serial_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         tmem_alloc(smem_u32(tmem_slot), 256);
         tmem_relinquish();
     }
-    load_rotate_q_tile(p, head, q0, sQ, tid, kSerialThreads);
+    load_rotate_q_tiles<kSerialThreads, 1>(p, head, q0, sQ, tid);
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();

@@ -69,6 +69,8 @@ struct MergeParams {
 
 // Launchers (each returns the launch error, enqueues on `stream`).
 cudaError_t launch_prep_kv(const PrepParams& p, cudaStream_t stream);
+cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
+                                  const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_merge_partials(const MergeParams& p, cudaStream_t stream);
 
 // Bytes of the partial-result scratch that follows K' and V't in the workspace: room for up to

@@ -10,28 +10,42 @@ namespace regenvc {
 constexpr uint32_t kTileBytes = kTile * kHeadDim * 2;  // 32 KB: one 128 x 128 16-bit tile
 constexpr uint32_t kBlockBytes = kTileBytes / 2;       // 16 KB: one [128][64] swizzled block
 
-// Loads a 128-row query tile, applies the rotary embedding and writes it to
-// shared memory as two swizzled K-major blocks (d 0..63, d 64..127).
-// Rows >= n_q are zero.  `nthreads` threads cooperate (multiple of 16).
-__device__ __forceinline__ void load_rotate_q_tile(const AttnParams& p, int head, int q0, uint8_t* sQ, int tid,
-                                                   int nthreads) {
+// Loads kTilesQ consecutive 128-row query tiles (rows q0 ..), applies the rotary embedding and writes each to
+// shared memory (sQ + tile * 32 KB) as two swizzled K-major fp16 blocks (d 0..63, d 64..127).  Rows >= n_q are
+// zero.  kThreadsN threads cooperate; every thread first issues all of its 16-byte global loads, then rotates
+// and stores, so that the loads overlap.
+template <int kThreadsN, int kTilesQ>
+__device__ __forceinline__ void load_rotate_q_tiles(const AttnParams& p, int head, int q0, uint8_t* sQ, int tid) {
+    static_assert(kThreadsN % 16 == 0 && (kTile * 16) % kThreadsN == 0, "thread count must tile the rows");
+    constexpr int kRowsPerPass = kThreadsN / 16;
+    constexpr int kPasses = kTile / kRowsPerPass;
     const int chunk = tid & 15;
-    for (int row = tid >> 4; row < kTile; row += nthreads >> 4) {
-        const int n = q0 + row;
-        uint4 packed = make_uint4(0, 0, 0, 0);
-        if (n < p.n_q) {
-            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)n * p.h + head) * kHeadDim) + chunk);
+    uint4 raw[kTilesQ][kPasses];
+#pragma unroll
+    for (int t = 0; t < kTilesQ; ++t)
+#pragma unroll
+        for (int it = 0; it < kPasses; ++it) {
+            const int n = q0 + t * kTile + it * kRowsPerPass + (tid >> 4);
+            raw[t][it] = make_uint4(0, 0, 0, 0);
+            if (n < p.n_q)
+                raw[t][it] = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)n * p.h + head) * kHeadDim) + chunk);
+        }
+#pragma unroll
+    for (int t = 0; t < kTilesQ; ++t)
+#pragma unroll
+        for (int it = 0; it < kPasses; ++it) {
+            const int row = it * kRowsPerPass + (tid >> 4);
+            const int n = q0 + t * kTile + row;
             float x[8];
-            bf16x8_to_float(raw, x);
-            if (p.rope) rope_rotate8(x, p.grid, token_pos(n, p.grid), chunk);
+            bf16x8_to_float(raw[t][it], x);
+            if (p.rope && n < p.n_q) rope_rotate8(x, p.grid, token_pos(n, p.grid), chunk);
+            uint4 packed;
             packed.x = pack_f16x2(x[0], x[1]);
             packed.y = pack_f16x2(x[2], x[3]);
             packed.z = pack_f16x2(x[4], x[5]);
             packed.w = pack_f16x2(x[6], x[7]);
+            *reinterpret_cast<uint4*>(sQ + t * kTileBytes + (chunk >> 3) * kBlockBytes + sw128_offset(row, chunk & 7)) = packed;
         }
-        *reinterpret_cast<uint4*>(sQ + (chunk >> 3) * kBlockBytes + sw128_offset(row, chunk & 7)) = packed;
-    }
 }
-
 
 }  // namespace regenvc
