@@ -103,6 +103,24 @@ class ClockSampler:
                 "power_w_max": max(self.power) if self.power else None}
 
 
+def rank_seed_offset(set_index: int, rank: int) -> int:
+    """Seed offset of input set `set_index` on `rank`: every rank runs its own window (distinct inputs)."""
+    return 100 * set_index + 7 * rank
+
+
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_tflops(world: int, flops_per_step: float, ms_per_step: float) -> float:
+    """Weak scaling: every rank processes one window per step; the job's rate is all windows over the slowest rank's time."""
+    return world * flops_per_step / (ms_per_step * 1e-3) / 1e12
+
+
 def step_flops(w: synth.Workload) -> float:
     return w.self_flops() + sum(w.cross_flops(n) for n in w.cross_kv)
 
@@ -198,7 +216,7 @@ def run_ours(args, w: synth.Workload):
     # inputs: N_BUFFER_SETS distinct sets so that consecutive steps do not find their inputs in L2
     sets = []
     for i in range(N_BUFFER_SETS):
-        wi = synth.Workload(**{**w.__dict__, "seed": w.seed + 100 * i + 7 * rank})
+        wi = synth.Workload(**{**w.__dict__, "seed": w.seed + rank_seed_offset(i, rank)})
         q, k, v = synth.self_inputs(wi)
         cross = [synth.cross_inputs(wi, n) for n in w.cross_kv]
         sets.append({"q": q.to(dev), "k": k.to(dev), "v": v.to(dev),
@@ -287,13 +305,10 @@ def run_ours(args, w: synth.Workload):
             e2e = {"ms": e2e_ms, "h2d": h2d, "d2h": d2h, "steps": n_e}
 
     # max over ranks
-    t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0, attn_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms, attn_ms_max = (float(x) for x in t.cpu())
+    ms_total, e2e_ms, attn_ms_max = max_over_ranks([ms_total, e2e["ms"] if e2e else 0.0, attn_ms], dist, dev)
     ms_step = ms_total / args.steps
     fl = step_flops(w)
-    value = world * fl / (ms_step * 1e-3) / 1e12
+    value = whole_job_tflops(world, fl, ms_step)
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
@@ -324,7 +339,7 @@ def run_ours(args, w: synth.Workload):
             "context": PAPER_CONTEXT,
         }
         if e2e:
-            line["e2e"] = {"value": world * fl / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+            line["e2e"] = {"value": whole_job_tflops(world, fl, e2e_ms), "unit": "TFLOP/s",
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                            "ms_per_step": e2e_ms, "steps": e2e["steps"]}
         if world == 1 and not args.no_cpu_baseline:
