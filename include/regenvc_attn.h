@@ -58,7 +58,8 @@ typedef enum {
     REGENVC_ERR_CUDA = 6,        /* a CUDA call failed: see regenvc_last_cuda_error() */
     REGENVC_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired (sticky device status) */
     REGENVC_ERR_WORKSPACE = 8,   /* caller-supplied workspace too small or misaligned */
-    REGENVC_ERR_RANGE = 9        /* an input exceeded the fp16 operand range (sticky device status) */
+    REGENVC_ERR_RANGE = 9,       /* an input exceeded the fp16 operand range (sticky device status) */
+    REGENVC_ERR_STATIC_LIMIT = 10 /* regenvc_cross_attn_forward_static(): the shape needs more than the built-in scratch */
 } regenvc_status;
 
 /*
@@ -95,6 +96,38 @@ int regenvc_attn_forward_host(const void* q, const void* k, const void* v, void*
                               float rope_theta, void* stream);
 int regenvc_cross_attn_forward_host(const void* q, const void* k, const void* v, void* out,
                                     int n_q, int n_kv, int n_heads, int head_dim, void* stream);
+
+/*
+ * Cross-attention for callers that must not allocate device memory.  (The paper has no counterpart: this
+ * is a deployment variant of regenvc_cross_attn_forward(), same arguments, same result.)
+ *
+ * Who needs it: code in the steady-state window loop of a real-time decoder.  cudaMalloc and cudaFree
+ * synchronise the whole device, so one allocation made on behalf of this library would stall the decode and
+ * encode streams running beside it and break the per-window time budget; and a serving process whose
+ * framework has already claimed nearly all device memory for its own pool may simply get an out-of-memory
+ * error from a raw cudaMalloc.  regenvc_cross_attn_forward() can do both on its first call or when its
+ * workspace has to grow.  This entry point never calls cudaMalloc, cudaFree or any allocating routine: the
+ * fp16 operand forms of k and v go into a fixed REGENVC_STATIC_SCRATCH_BYTES array that is part of the
+ * library image, so every GPU that loads the library holds those bytes until the process exits.
+ *
+ *   - Limit: 2 * n_heads * n_kv_pad * 256 bytes (n_kv_pad = n_kv rounded up to 128) must fit in the array,
+ *     i.e. n_heads * n_kv_pad <= 32768 (12 heads x 2688 keys, 40 heads x 768 keys).  Larger shapes are
+ *     rejected with REGENVC_ERR_STATIC_LIMIT and nothing is enqueued.  The key range is never cut into
+ *     pieces here (that path needs extra scratch), so very long conditioning sequences run slower than
+ *     through regenvc_cross_attn_forward().
+ *   - The first call on each device looks up the device address of the array (and sets kernel attributes);
+ *     make that call during start-up, before any stream capture is begun.
+ *   - All calls on a device share the one array, which still holds the previous call's operands when the
+ *     next call starts.  Each call rewrites everything it later reads (padding rows included), so nothing
+ *     needs clearing between calls; but two calls that overlap on the GPU (different streams, or different
+ *     host threads) race on the array and give wrong results: keep them on one stream or order them with
+ *     events.  regenvc_set_workspace() has no effect here.
+ *   - Device-side conditions of these calls (an input beyond the fp16 range, an expired bounded wait) are
+ *     recorded in a status word that is also part of the image, not in the one regenvc_device_status() reads.
+ */
+#define REGENVC_STATIC_SCRATCH_BYTES (16u << 20)
+int regenvc_cross_attn_forward_static(const void* q, const void* k, const void* v, void* out,
+                                      int n_q, int n_kv, int n_heads, int head_dim, void* stream);
 
 /*
  * Scratch memory.  Each call first rewrites the keys and values into

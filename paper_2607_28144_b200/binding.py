@@ -16,13 +16,15 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libregenvc_attn.so")
 
 OK, ERR_NULL_POINTER, ERR_BAD_SHAPE, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_ALIASING, ERR_CUDA, ERR_TIMEOUT, \
-    ERR_WORKSPACE, ERR_RANGE = range(10)
+    ERR_WORKSPACE, ERR_RANGE, ERR_STATIC_LIMIT = range(11)
+STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = [
     "regenvc_attn_forward", "regenvc_cross_attn_forward", "regenvc_attn_forward_host",
     "regenvc_cross_attn_forward_host", "regenvc_workspace_bytes", "regenvc_set_workspace",
     "regenvc_device_status", "regenvc_status_string", "regenvc_last_cuda_error", "regenvc_version",
     "regenvc_kernel_launch_count", "regenvc_shutdown", "regenvc_debug_set_phases",
+    "regenvc_cross_attn_forward_static",
 ]
 
 _lib = None
@@ -48,6 +50,8 @@ def lib() -> ctypes.CDLL:
     L.regenvc_attn_forward.restype = i32
     L.regenvc_cross_attn_forward.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
     L.regenvc_cross_attn_forward.restype = i32
+    L.regenvc_cross_attn_forward_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+    L.regenvc_cross_attn_forward_static.restype = i32
     L.regenvc_attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, vp]
     L.regenvc_attn_forward_host.restype = i32
     L.regenvc_cross_attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
@@ -124,6 +128,22 @@ def regenvc_cross_attn_forward(q, k, v, out, stream=None):
         raise ValueError("shape mismatch")
     _check(lib().regenvc_cross_attn_forward(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), n_q, n_kv, h, d,
                                             _stream(stream)))
+    return out
+
+
+def regenvc_cross_attn_forward_static(q, k, v, out, stream=None):
+    """Cross-attention without any device allocation by the library (for callers in a real-time loop, or
+    in a process whose memory pool owns the GPU): the operand scratch is a fixed 16 MiB array inside the
+    library, shared by all calls on the device, so calls must not overlap on the GPU; shapes with
+    n_heads * ceil(n_kv / 128) * 128 > 32768 raise ERR_STATIC_LIMIT."""
+    for t, nm in ((q, "q"), (k, "k"), (v, "v"), (out, "out")):
+        _dev_bf16(t, nm)
+    n_q, h, d = q.shape
+    n_kv = k.shape[0]
+    if k.shape != (n_kv, h, d) or v.shape != k.shape or out.shape != q.shape:
+        raise ValueError("shape mismatch")
+    _check(lib().regenvc_cross_attn_forward_static(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), n_q,
+                                                   n_kv, h, d, _stream(stream)))
     return out
 
 

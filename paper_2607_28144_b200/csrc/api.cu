@@ -443,6 +443,7 @@ const char* regenvc_status_string(int status) {
         case REGENVC_ERR_TIMEOUT: return "device-side bounded wait expired";
         case REGENVC_ERR_WORKSPACE: return "workspace too small or misaligned";
         case REGENVC_ERR_RANGE: return "input outside the fp16 operand range";
+        case REGENVC_ERR_STATIC_LIMIT: return "shape exceeds the built-in scratch of the allocation-free entry point";
         default: return "unknown status";
     }
 }

@@ -71,6 +71,7 @@ struct MergeParams {
 cudaError_t launch_prep_kv(const PrepParams& p, cudaStream_t stream);
 cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
                                   const AttnParams& p, cudaStream_t stream);
+cudaError_t configure_attn_pipelined();   // once per device: register hand-over check, large dynamic shared memory
 cudaError_t launch_merge_partials(const MergeParams& p, cudaStream_t stream);
 
 // Bytes of the partial-result scratch that follows K' and V't in the workspace: room for up to

@@ -26,7 +26,7 @@ def _declared_symbols():
 
 def test_every_declared_symbol_is_exported(L):
     declared = _declared_symbols()
-    assert len(declared) >= 12
+    assert len(declared) >= 14
     for name in declared:
         assert hasattr(L, name), f"{name} declared in the header but not exported"
     assert sorted(binding.EXPORTS) == [d for d in declared if d in binding.EXPORTS]
@@ -35,8 +35,8 @@ def test_every_declared_symbol_is_exported(L):
 
 def test_status_strings_and_version(L):
     assert binding.regenvc_version().startswith("regenvc-attn")
-    seen = {binding.status_string(c) for c in range(10)}
-    assert len(seen) == 10 and binding.status_string(99) == "unknown status"
+    seen = {binding.status_string(c) for c in range(11)}
+    assert len(seen) == 11 and binding.status_string(99) == "unknown status"
 
 
 def test_workspace_bytes():
