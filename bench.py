@@ -36,9 +36,9 @@ NOMINAL_BF16_TFLOPS = 2250.0  # dense bf16/fp16 datasheet figure, context only
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 PAPER_CONTEXT = ("paper: 972 ms per 25-frame window (24 fps) for the WHOLE decoder on 8 consumer-class GPUs; "
                  "it reports no attention-only number")
-# DRAM bytes per launch of the attention kernel at the 480x832 window shape, from the ncu capture
-# summarised in profiles/ (None until a capture exists).
-ATTN_KERNEL_DRAM_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the self-attention kernel at the 480x832 window
+# shape, from the ncu capture summarised in profiles/attn_pipelined_kernel_window_480x832.md (101.5 MB + 19.1 MB).
+ATTN_KERNEL_DRAM_TRAFFIC_BYTES = {"window_480x832": 120.6e6}
 N_BUFFER_SETS = 4
 
 
@@ -335,7 +335,8 @@ def run_ours(args, w: synth.Workload):
                          "frac_of_burst": achieved / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"])),
                          "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
                          "kernel_ms_mean": attn_ms, "kernel_ms_best": attn_ms_best, "prep_kernel_ms": prep_ms,
-                         "traffic": ATTN_KERNEL_DRAM_TRAFFIC_BYTES},
+                         "traffic": ATTN_KERNEL_DRAM_TRAFFIC_BYTES.get(w.name),
+                         "algorithmic_hbm_bytes": 4.0 * w.n_tokens * w.n_heads * 256},
             "context": PAPER_CONTEXT,
         }
         if e2e:
