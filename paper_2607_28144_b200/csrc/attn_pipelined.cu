@@ -66,6 +66,9 @@ constexpr int kSoftmaxRegs = ((kLaunchRegs * kThreads - kControlRegs * 128) / kS
 static_assert(kSoftmaxRegs * kSoftmaxThreads + kControlRegs * 128 <= kLaunchRegs * kThreads, "register budget");
 static_assert(kSoftmaxRegs >= kLaunchRegs && kSoftmaxRegs <= 255, "setmaxnreg.inc must not shrink");
 constexpr int kMmaWarp = kSoftmaxThreads / 32, kTmaWarp = kMmaWarp + 1;
+#ifndef REGENVC_EXP_F16
+#define REGENVC_EXP_F16 0
+#endif
 #ifndef REGENVC_POLY_MASK
 #define REGENVC_POLY_MASK 0x52
 #endif
@@ -151,6 +154,29 @@ __device__ __forceinline__ void exp_chunk(const uint32_t* s, uint64_t scale2, ui
     }
 }
 
+// Half-precision variant: x = s * scale - m_ref is formed in fp32, rounded to fp16 and exponentiated two at a
+// time by the MUFU's packed fp16 ex2, whose result already is the fp16 operand P; the part's row sum is a short
+// fp16 tree (16 terms per half) widened to fp32.  Rounding x to fp16 perturbs each probability by up to
+// ~0.3 % at |x| ~ 16 (less for the large ones), without bias, and the row sum is taken over the very values
+// that enter P.V, so the perturbations average out over the keys of a row.
+__device__ __forceinline__ float exp_chunk_h2(const uint32_t* s, uint64_t scale2, uint64_t negm2, uint32_t* pr) {
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        const uint64_t x2 = fma2(pack2(__uint_as_float(s[2 * c]), __uint_as_float(s[2 * c + 1])), scale2, negm2);
+        float x0, x1;
+        unpack2(x2, x0, x1);
+        pr[c] = ex2_f16x2(pack_f16x2(x0, x1));
+    }
+    uint32_t t[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) t[c] = add_f16x2(pr[2 * c], pr[2 * c + 1]);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) t[c] = add_f16x2(t[2 * c], t[2 * c + 1]);
+    t[0] = add_f16x2(t[0], t[1]);
+    t[2] = add_f16x2(t[2], t[3]);
+    return sum_halves_f16x2(add_f16x2(t[0], t[2]));
+}
+
 // The eight K = 16 steps of one 128 x 128 x 128 product.  Descriptors differ only in the start-address
 // field: +2 (32 bytes) per K step inside a 128-byte row, +1024 (16 KB) for the second 64-element block.
 __device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint32_t sQ, uint32_t sK) {
@@ -231,6 +257,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
 
     if (tid == 0) TRACE_CTA(1);
     const uint32_t tmem_base = bar->tmem_base;
+    const uint32_t xch_base = smem_u32(&xch->v[0][0][0][0]);
     const WaitCtl ctl{&bar->abort_flag, p.status, kStatusTimeout, kWaitLimitNs};
 
     if (warp >= kMmaWarp) {
@@ -338,6 +365,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                                   part * kColsPerThread;
                 uint64_t negm2 = pack2(-m_ref[t], -m_ref[t]);
                 uint64_t sum_a = 0, sum_b = 0;  // packed partial row sums
+                float h2_sum = 0.f;
                 const bool stream = j > 0;
                 if (ok) {
                     tmem_ld32(t_S, sr);
@@ -352,7 +380,11 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                         }
                         if (stream) {
                             uint32_t pr[16];
+#if REGENVC_EXP_F16
+                            h2_sum += exp_chunk_h2(sr + cb * 32, scale2, negm2, pr);
+#else
                             exp_chunk<kPolyMask>(sr + cb * 32, scale2, negm2, pr, sum_a, sum_b);
+#endif
                             tmem_st16(t_S + cb * 16, pr);
                         }
                     }
@@ -361,13 +393,18 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 {
                     float s0, s1;
                     unpack2(add2(sum_a, sum_b), s0, s1);
-                    part_sum = s0 + s1;
+                    part_sum = s0 + s1 + h2_sum;
                 }
-                xch->v[j & 1][t][row][part] = part_sum;
+                const uint32_t xrow = xch_base + static_cast<uint32_t>((((j & 1) * 2 + t) * kTile + row) * kSplit * sizeof(float));
+                sts_f32(xrow + part * sizeof(float), part_sum);
                 row_group_barrier(warp & 3);
-                bool redo = !stream || !(part_sum < 65504.0f);
-#pragma unroll
-                for (int o = 1; o < kSplit; ++o) redo |= !(xch->v[j & 1][t][row][(part + o) % kSplit] < 65504.0f);
+                bool redo = !stream;
+                if (kSplit == 4) {
+                    const float4 sums = lds_f32x4(xrow);  // the four parts of this row (own one included)
+                    redo |= !(fmaxf(fmaxf(sums.x, sums.y), fmaxf(sums.z, sums.w)) < 65504.0f);
+                } else {
+                    redo |= !(fmaxf(part_sum, lds_f32(xrow + (part ^ 1) * sizeof(float))) < 65504.0f);
+                }
                 if (tid == 0) TRACE(j, t * 6 + 2);
                 const bool any_redo = __any_sync(0xffffffffu, redo);
                 if (any_redo) {
@@ -412,18 +449,23 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     negm2 = pack2(-m_ref[t], -m_ref[t]);
                     sum_a = 0;
                     sum_b = 0;
+                    h2_sum = 0.f;
                     if (ok) {
 #pragma unroll
                         for (int cb = 0; cb < kChunks; ++cb) {
                             uint32_t pr[16];
+#if REGENVC_EXP_F16
+                            h2_sum += exp_chunk_h2(sr + cb * 32, scale2, negm2, pr);
+#else
                             exp_chunk<kPolyMask>(sr + cb * 32, scale2, negm2, pr, sum_a, sum_b);
+#endif
                             tmem_st16(t_S + cb * 16, pr);
                         }
                     }
                 }
                 float s0, s1;
                 unpack2(add2(sum_a, sum_b), s0, s1);
-                l_run[t] += s0 + s1;
+                l_run[t] += s0 + s1 + h2_sum;
                 if (tid == 0) TRACE(j, t * 6 + 3);
                 tmem_wait_st();
                 tc_fence_before();
