@@ -70,7 +70,7 @@ constexpr int kMmaWarp = kSoftmaxThreads / 32, kTmaWarp = kMmaWarp + 1;
 #define REGENVC_EXP_F16 0
 #endif
 #ifndef REGENVC_POLY_MASK
-#define REGENVC_POLY_MASK 0x52
+#define REGENVC_POLY_MASK 0x44
 #endif
 // bit i set: pair i of every eight probability pairs takes the polynomial 2^x instead of the MUFU
 constexpr uint32_t kPolyMask = REGENVC_POLY_MASK;
