@@ -8,12 +8,18 @@
 // of the ~N/128 query-tile CTAs that stream it.  HBM-bound: 2 x 256 B read and
 // 2 x 256 B written per (token, head).
 #include "common.cuh"
+#include "ptx.cuh"
 #include "rope.cuh"
 
 namespace regenvc {
 
 constexpr int kPrepThreads = 256;
-constexpr int kVtStride = 65;  // words per d-row of the transpose tile (64 token pairs + 1 pad)
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
 
 __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
     const int tid = threadIdx.x;
@@ -21,68 +27,81 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
     const int head = blockIdx.y;
 
     if (blockIdx.z == 0) {
-        // ---- K: 16 threads per row (16 B = 8 elements = 4 rotary pairs each)
+        // ---- K: 16 threads per row (16 B = 8 elements = 4 rotary pairs each); all loads first
         const int chunk = tid & 15;
         bool out_of_range = false;
-#pragma unroll 2
+        uint4 raw[kTile / 16];
+#pragma unroll
         for (int it = 0; it < kTile / 16; ++it) {
             const int n = tile0 + it * 16 + (tid >> 4);
-            uint4 packed = make_uint4(0, 0, 0, 0);
-            if (n < p.n_kv) {
-                const uint4 raw =
-                    __ldg(reinterpret_cast<const uint4*>(p.k + ((size_t)n * p.h + head) * kHeadDim) + chunk);
-                float x[8];
-                bf16x8_to_float(raw, x);
-                if (p.rope) rope_rotate8(x, p.grid, token_pos(n, p.grid), chunk);
-                __half2 h0 = __floats2half2_rn(x[0], x[1]);
-                __half2 h1 = __floats2half2_rn(x[2], x[3]);
-                __half2 h2 = __floats2half2_rn(x[4], x[5]);
-                __half2 h3 = __floats2half2_rn(x[6], x[7]);
+            raw[it] = make_uint4(0, 0, 0, 0);
+            if (n < p.n_kv)
+                raw[it] = __ldg(reinterpret_cast<const uint4*>(p.k + ((size_t)n * p.h + head) * kHeadDim) + chunk);
+        }
 #pragma unroll
-                for (int i = 0; i < 8; ++i) out_of_range |= !(fabsf(x[i]) <= 65504.0f);
-                packed.x = *reinterpret_cast<uint32_t*>(&h0);
-                packed.y = *reinterpret_cast<uint32_t*>(&h1);
-                packed.z = *reinterpret_cast<uint32_t*>(&h2);
-                packed.w = *reinterpret_cast<uint32_t*>(&h3);
-            }
+        for (int it = 0; it < kTile / 16; ++it) {
+            const int n = tile0 + it * 16 + (tid >> 4);
+            float x[8];
+            bf16x8_to_float(raw[it], x);
+            if (p.rope && n < p.n_kv) rope_rotate8(x, p.grid, token_pos(n, p.grid), chunk);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) out_of_range |= !(fabsf(x[i]) <= 65504.0f);
+            uint4 packed;
+            packed.x = pack_f16x2(x[0], x[1]);
+            packed.y = pack_f16x2(x[2], x[3]);
+            packed.z = pack_f16x2(x[4], x[5]);
+            packed.w = pack_f16x2(x[6], x[7]);
             reinterpret_cast<uint4*>(p.kp + ((size_t)head * p.n_kv_pad + n) * kHeadDim)[chunk] = packed;
         }
         if (out_of_range) atomicCAS(p.status, 0, kStatusRange);
     } else {
         // ---- V: transpose a [128 tokens][128 d] tile through shared memory.
-        // tile[d][tp] holds the fp16 pair (token 2*tp, token 2*tp+1) of column d.
-        __shared__ uint32_t tile[kHeadDim * kVtStride];
+        // tile[d][tp ^ swz(d)] holds the fp16 pair (token 2*tp, token 2*tp+1) of column d; swz(d) = (d / 4) % 32
+        // makes both the column-wise writes below and the row-wise reads conflict-free.
+        __shared__ uint32_t tile[kHeadDim * 64];
         const int warp = tid >> 5, lane = tid & 31;
+        const int tb = lane >> 4, c = lane & 15;  // token of the pair, 8-column chunk
         bool out_of_range = false;
+        uint4 raw[8];
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int n = tile0 + 2 * (warp * 8 + it) + tb;
+            raw[it] = make_uint4(0, 0, 0, 0);
+            if (n < p.n_kv)
+                raw[it] = __ldg(reinterpret_cast<const uint4*>(p.v + ((size_t)n * p.h + head) * kHeadDim) + c);
+        }
+#pragma unroll
         for (int it = 0; it < 8; ++it) {
             const int tp = warp * 8 + it;
-            const int n0 = tile0 + 2 * tp;
+            float x[8];
+            bf16x8_to_float(raw[it], x);
 #pragma unroll
-            for (int half_row = 0; half_row < 2; ++half_row) {
-                const int d = half_row * 64 + 2 * lane;
-                uint32_t a = 0, b = 0;  // (v[n0][d], v[n0][d+1]) and the same for n0+1, as bf16 pairs
-                if (n0 < p.n_kv)
-                    a = __ldg(reinterpret_cast<const uint32_t*>(p.v + ((size_t)n0 * p.h + head) * kHeadDim + d));
-                if (n0 + 1 < p.n_kv)
-                    b = __ldg(reinterpret_cast<const uint32_t*>(p.v + ((size_t)(n0 + 1) * p.h + head) * kHeadDim + d));
-                const float a0 = __uint_as_float(a << 16), a1 = __uint_as_float(a & 0xffff0000u);
-                const float b0 = __uint_as_float(b << 16), b1 = __uint_as_float(b & 0xffff0000u);
-                out_of_range |= !(fabsf(a0) <= 65504.0f) | !(fabsf(a1) <= 65504.0f) | !(fabsf(b0) <= 65504.0f) |
-                                !(fabsf(b1) <= 65504.0f);
-                __half2 c0 = __floats2half2_rn(a0, b0);  // column d:   tokens n0, n0+1
-                __half2 c1 = __floats2half2_rn(a1, b1);  // column d+1
-                tile[d * kVtStride + tp] = *reinterpret_cast<uint32_t*>(&c0);
-                tile[(d + 1) * kVtStride + tp] = *reinterpret_cast<uint32_t*>(&c1);
-            }
+            for (int i = 0; i < 8; ++i) out_of_range |= !(fabsf(x[i]) <= 65504.0f);
+            const uint32_t h0 = pack_f16x2(x[0], x[1]), h1 = pack_f16x2(x[2], x[3]);
+            const uint32_t h2 = pack_f16x2(x[4], x[5]), h3 = pack_f16x2(x[6], x[7]);
+            // the lane of token 0 keeps columns 0..3 of the chunk, the lane of token 1 columns 4..7
+            const uint32_t recv_a = __shfl_xor_sync(0xffffffffu, tb ? h0 : h2, 16);
+            const uint32_t recv_b = __shfl_xor_sync(0xffffffffu, tb ? h1 : h3, 16);
+            const uint32_t mine_a = tb ? h2 : h0, mine_b = tb ? h3 : h1;
+            const uint32_t lo_a = tb ? recv_a : mine_a, hi_a = tb ? mine_a : recv_a;  // token 0 / token 1
+            const uint32_t lo_b = tb ? recv_b : mine_b, hi_b = tb ? mine_b : recv_b;
+            const int d0 = 8 * c + 4 * tb;
+            const int col = tp ^ ((d0 >> 2) & 31);
+            tile[(d0 + 0) * 64 + col] = prmt(lo_a, hi_a, 0x5410);
+            tile[(d0 + 1) * 64 + col] = prmt(lo_a, hi_a, 0x7632);
+            tile[(d0 + 2) * 64 + col] = prmt(lo_b, hi_b, 0x5410);
+            tile[(d0 + 3) * 64 + col] = prmt(lo_b, hi_b, 0x7632);
         }
         if (out_of_range) atomicCAS(p.status, 0, kStatusRange);
         __syncthreads();
         uint32_t* dst = reinterpret_cast<uint32_t*>(p.vt + (size_t)head * kHeadDim * p.n_kv_pad + tile0);
         const size_t row_words = (size_t)p.n_kv_pad / 2;
-        for (int it = 0; it < kHeadDim / 8; ++it) {
-            const int d = it * 8 + warp;
-            dst[d * row_words + lane] = tile[d * kVtStride + lane];
-            dst[d * row_words + 32 + lane] = tile[d * kVtStride + 32 + lane];
+#pragma unroll 4
+        for (int r = 0; r < kHeadDim / 8; ++r) {
+            const int d = warp * (kHeadDim / 8) + r;
+            const int swz = (d >> 2) & 31;
+            dst[d * row_words + lane] = tile[d * 64 + (lane ^ swz)];
+            dst[d * row_words + 32 + lane] = tile[d * 64 + 32 + (lane ^ swz)];
         }
     }
 }
