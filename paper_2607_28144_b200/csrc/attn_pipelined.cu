@@ -29,22 +29,6 @@
 
 namespace regenvc {
 
-#ifdef REGENVC_TRACE
-// Bring-up instrumentation (never compiled into the shipped library): clock64 stamps of one CTA.
-__device__ long long g_trace[64 * 32];
-#define TRACE(j, slot)                                                                  \
-    do {                                                                                \
-        if (blockIdx.x == 3 && (j) >= 16 && (j) < 80)                \
-            g_trace[((j) - 16) * 32 + (slot)] = clock64();                              \
-    } while (0)
-#define TRACE_CTA(slot)                                                                 \
-    do {                                                                                \
-        if (blockIdx.x == 3) g_trace[63 * 32 + (slot)] = clock64();                     \
-    } while (0)
-#else
-#define TRACE(j, slot) do {} while (0)
-#define TRACE_CTA(slot) do {} while (0)
-#endif
 
 namespace {
 
@@ -66,9 +50,6 @@ constexpr int kSoftmaxRegs = ((kLaunchRegs * kThreads - kControlRegs * 128) / kS
 static_assert(kSoftmaxRegs * kSoftmaxThreads + kControlRegs * 128 <= kLaunchRegs * kThreads, "register budget");
 static_assert(kSoftmaxRegs >= kLaunchRegs && kSoftmaxRegs <= 255, "setmaxnreg.inc must not shrink");
 constexpr int kMmaWarp = kSoftmaxThreads / 32, kTmaWarp = kMmaWarp + 1;
-#ifndef REGENVC_EXP_F16
-#define REGENVC_EXP_F16 0
-#endif
 #ifndef REGENVC_POLY_MASK
 #define REGENVC_POLY_MASK 0x44
 #endif
@@ -123,6 +104,20 @@ __device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
 __device__ __forceinline__ void softmax_barrier() {
     asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
 }
+// The same barrier with an OR-reduction of one predicate per thread: every thread of the row group learns
+// whether any of them raised the flag, without touching shared memory.
+__device__ __forceinline__ bool row_group_any(int g, bool flag) {
+    uint32_t any;
+    asm volatile(
+        "{\n\t.reg .pred pin, pout;\n\t"
+        "setp.ne.u32 pin, %1, 0;\n\t"
+        "bar.red.or.pred pout, %2, %3, pin;\n\t"
+        "selp.u32 %0, 1, 0, pout;\n\t}"
+        : "=r"(any)
+        : "r"(static_cast<uint32_t>(flag)), "r"(2 + g), "n"(32 * kSplit)
+        : "memory");
+    return any != 0;
+}
 // Named barrier over the kSplit warps that share the 32 rows of lane group g (barriers 2..5).
 __device__ __forceinline__ void row_group_barrier(int g) {
     asm volatile("bar.sync %0, %1;" ::"r"(2 + g), "n"(32 * kSplit) : "memory");
@@ -152,29 +147,6 @@ __device__ __forceinline__ void exp_chunk(const uint32_t* s, uint64_t scale2, ui
         unpack2(p2, p0, p1);
         pr[c] = pack_f16x2_sat(p0, p1);
     }
-}
-
-// Half-precision variant: x = s * scale - m_ref is formed in fp32, rounded to fp16 and exponentiated two at a
-// time by the MUFU's packed fp16 ex2, whose result already is the fp16 operand P; the part's row sum is a short
-// fp16 tree (16 terms per half) widened to fp32.  Rounding x to fp16 perturbs each probability by up to
-// ~0.3 % at |x| ~ 16 (less for the large ones), without bias, and the row sum is taken over the very values
-// that enter P.V, so the perturbations average out over the keys of a row.
-__device__ __forceinline__ float exp_chunk_h2(const uint32_t* s, uint64_t scale2, uint64_t negm2, uint32_t* pr) {
-#pragma unroll
-    for (int c = 0; c < 16; ++c) {
-        const uint64_t x2 = fma2(pack2(__uint_as_float(s[2 * c]), __uint_as_float(s[2 * c + 1])), scale2, negm2);
-        float x0, x1;
-        unpack2(x2, x0, x1);
-        pr[c] = ex2_f16x2(pack_f16x2(x0, x1));
-    }
-    uint32_t t[8];
-#pragma unroll
-    for (int c = 0; c < 8; ++c) t[c] = add_f16x2(pr[2 * c], pr[2 * c + 1]);
-#pragma unroll
-    for (int c = 0; c < 4; ++c) t[c] = add_f16x2(t[2 * c], t[2 * c + 1]);
-    t[0] = add_f16x2(t[0], t[1]);
-    t[2] = add_f16x2(t[2], t[3]);
-    return sum_halves_f16x2(add_f16x2(t[0], t[2]));
 }
 
 // The eight K = 16 steps of one 128 x 128 x 128 product.  Descriptors differ only in the start-address
@@ -226,7 +198,6 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     const int q0 = (item % p.pairs_per_head) * 2 * kTile;
     const bool tile1_active = q0 + kTile < p.n_q;
 
-    if (tid == 0) TRACE_CTA(0);
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_u32(&bar->kv_full[s]), 1);
@@ -255,9 +226,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     __syncthreads();
     tc_fence_after();
 
-    if (tid == 0) TRACE_CTA(1);
     const uint32_t tmem_base = bar->tmem_base;
-    const uint32_t xch_base = smem_u32(&xch->v[0][0][0][0]);
     const WaitCtl ctl{&bar->abort_flag, p.status, kStatusTimeout, kWaitLimitNs};
 
     if (warp >= kMmaWarp) {
@@ -308,15 +277,12 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     ok = mbar_wait(smem_u32(&bar->p_full[t]), j & 1, ctl);
                     if (!ok) break;
                     tc_fence_after();
-                    TRACE(j, 12 + t * 2);
                     issue_pv(tmem_base + 256 + t * 128, tmem_base + t * 128, smem_u32(sKV + slot_v * kTileBytes), j > 0);
                     umma_commit(smem_u32(&bar->o_full[t]));
-                    TRACE(j, 5 + t * 6);
                     if (more) {
                         issue_qk(tmem_base + t * 128, t ? sQ1 : sQ0, smem_u32(sKV + slot_k * kTileBytes));
                         umma_commit(smem_u32(&bar->s_full[t]));
                     }
-                    TRACE(j, 13 + t * 2);
                 }
                 if (ok) {
                     umma_commit(smem_u32(&bar->kv_empty[slot_v]));
@@ -335,12 +301,15 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         else load_rotate_q_tiles<kSoftmaxThreads, 1>(p, head, q0, sQ, tid);
         fence_proxy_async_smem();
         for (int t = 0; t < n_active; ++t) mbar_arrive(smem_u32(&bar->q_full[t]));
-        if (tid == 0) TRACE_CTA(2);
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         const float scale = p.scale_log2;
         const uint64_t scale2 = pack2(scale, scale);
         float m_ref[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
         bool ok = true;  // false once a wait expired: keep the loop structure (named barriers) but skip the work
+        // the one key tile of the sequence that is partly padding (if this CTA has it), and how many of this
+        // thread's columns of that tile are real keys
+        const int j_ragged = (p.n_kv % kTile != 0 && kv_tile0 + n_tiles == n_tiles_total) ? n_tiles - 1 : -1;
+        const int valid_last = p.n_kv - (n_tiles_total - 1) * kTile - part * kColsPerThread;
 
         for (int j = 0; j < n_tiles; ++j) {
 #pragma unroll
@@ -348,24 +317,17 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 if (t >= n_active) continue;
                 const uint32_t t_S = lane_base + t * 128 + part * kColsPerThread;
                 const uint32_t t_O = lane_base + 256 + t * 128 + part * kColsPerThread;
-                if (tid == 0) TRACE(j, t * 6 + 0);
                 if (ok) ok = mbar_wait(smem_u32(&bar->s_full[t]), j & 1, ctl);
                 ok = __all_sync(0xffffffffu, ok);  // keep the warp-wide TMEM instructions below convergent
                 tc_fence_after();
-                if (tid == 0) TRACE(j, t * 6 + 1);
-                if (tid == 0 && j == 0 && t == 0) TRACE_CTA(3);
                 // From the second tile on, the probabilities of each 32-column chunk are formed as soon as it
                 // arrives, against the reference m_ref of the earlier tiles; no maximum is taken.  Probabilities
                 // saturate at 65504 when rounded to fp16, and a saturated one makes the fp32 sum of its part reach
                 // 65504, which the threads of the row detect by exchanging their sums; only then (and on the first
                 // tile) the row maximum is taken, the reference raised, O rescaled and the tile redone.
                 uint32_t sr[kColsPerThread];
-                // own columns >= valid are padding
-                const int valid = ((kv_tile0 + j == n_tiles_total - 1) ? p.n_kv - (kv_tile0 + j) * kTile : kTile) -
-                                  part * kColsPerThread;
                 uint64_t negm2 = pack2(-m_ref[t], -m_ref[t]);
                 uint64_t sum_a = 0, sum_b = 0;  // packed partial row sums
-                float h2_sum = 0.f;
                 const bool stream = j > 0;
                 if (ok) {
                     tmem_ld32(t_S, sr);
@@ -373,18 +335,14 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     for (int cb = 0; cb < kChunks; ++cb) {
                         tmem_wait_ld();
                         if (cb + 1 < kChunks) tmem_ld32(t_S + 32 * (cb + 1), sr + 32 * (cb + 1));
-                        if (valid < kColsPerThread) {
+                        if (j == j_ragged) {  // the sequence's last, partly padded key tile
 #pragma unroll
                             for (int c = 0; c < 32; ++c)
-                                if (cb * 32 + c >= valid) sr[cb * 32 + c] = 0xff800000u;  // -inf
+                                if (cb * 32 + c >= valid_last) sr[cb * 32 + c] = 0xff800000u;  // -inf
                         }
                         if (stream) {
                             uint32_t pr[16];
-#if REGENVC_EXP_F16
-                            h2_sum += exp_chunk_h2(sr + cb * 32, scale2, negm2, pr);
-#else
                             exp_chunk<kPolyMask>(sr + cb * 32, scale2, negm2, pr, sum_a, sum_b);
-#endif
                             tmem_st16(t_S + cb * 16, pr);
                         }
                     }
@@ -393,24 +351,15 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 {
                     float s0, s1;
                     unpack2(add2(sum_a, sum_b), s0, s1);
-                    part_sum = s0 + s1 + h2_sum;
+                    part_sum = s0 + s1;
                 }
-                const uint32_t xrow = xch_base + static_cast<uint32_t>((((j & 1) * 2 + t) * kTile + row) * kSplit * sizeof(float));
-                sts_f32(xrow + part * sizeof(float), part_sum);
-                row_group_barrier(warp & 3);
-                bool redo = !stream;
-                if (kSplit == 4) {
-                    const float4 sums = lds_f32x4(xrow);  // the four parts of this row (own one included)
-                    redo |= !(fmaxf(fmaxf(sums.x, sums.y), fmaxf(sums.z, sums.w)) < 65504.0f);
-                } else {
-                    redo |= !(fmaxf(part_sum, lds_f32(xrow + (part ^ 1) * sizeof(float))) < 65504.0f);
-                }
-                if (tid == 0) TRACE(j, t * 6 + 2);
-                const bool any_redo = __any_sync(0xffffffffu, redo);
+                // One barrier with an OR-reduction tells the threads sharing these 32 rows whether any part of any
+                // row saturated (or this is the first tile); only then do they exchange anything.
+                const bool any_redo = row_group_any(warp & 3, !stream || !(part_sum < 65504.0f));
                 if (any_redo) {
-                    // Rare after the first tile.  The warps sharing these rows see the same flags and take the
-                    // same branch: row maximum, new reference for the flagged rows, rescale of this thread's part
-                    // of the O row and of its row sum, then the probabilities of the tile against the reference.
+                    // Rare after the first tile.  All threads of the row group take this branch together: row
+                    // maximum, a higher reference for the rows whose maximum exceeds theirs, rescale of this
+                    // thread's part of the O row and of its row sum, then the probabilities against the reference.
                     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
                     for (int c = 0; c < kColsPerThread; c += 8) {
@@ -427,11 +376,12 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     for (int o = 1; o < kSplit; ++o) mx_row = fmaxf(mx_row, xch->m[t][row][(part + o) % kSplit]);
                     row_group_barrier(warp & 3);  // everyone has read xch->m before a later redo overwrites it
                     const float m_tile = mx_row * scale;
+                    const bool raise = m_tile > m_ref[t];  // always on the first tile (reference starts at -inf)
                     if (j > 0) {
                         if (ok) ok = mbar_wait(smem_u32(&bar->o_full[t]), (j - 1) & 1, ctl);
                         ok = __all_sync(0xffffffffu, ok);
                         tc_fence_after();
-                        const float alpha = redo ? ex2_approx(m_ref[t] - m_tile) : 1.0f;
+                        const float alpha = raise ? ex2_approx(m_ref[t] - m_tile) : 1.0f;
                         l_run[t] *= alpha;
                         if (ok) {
 #pragma unroll 1
@@ -445,36 +395,27 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                             }
                         }
                     }
-                    if (redo) m_ref[t] = m_tile;
+                    if (raise) m_ref[t] = m_tile;
                     negm2 = pack2(-m_ref[t], -m_ref[t]);
                     sum_a = 0;
                     sum_b = 0;
-                    h2_sum = 0.f;
                     if (ok) {
 #pragma unroll
                         for (int cb = 0; cb < kChunks; ++cb) {
                             uint32_t pr[16];
-#if REGENVC_EXP_F16
-                            h2_sum += exp_chunk_h2(sr + cb * 32, scale2, negm2, pr);
-#else
                             exp_chunk<kPolyMask>(sr + cb * 32, scale2, negm2, pr, sum_a, sum_b);
-#endif
                             tmem_st16(t_S + cb * 16, pr);
                         }
                     }
                 }
                 float s0, s1;
                 unpack2(add2(sum_a, sum_b), s0, s1);
-                l_run[t] += s0 + s1 + h2_sum;
-                if (tid == 0) TRACE(j, t * 6 + 3);
+                l_run[t] += s0 + s1;
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bar->p_full[t]));
-                if (tid == 0) TRACE(j, t * 6 + 4);
-                if (tid == 0 && j == 0 && t == 0) TRACE_CTA(4);
             }
         }
-        if (tid == 0) TRACE_CTA(5);
 
         // epilogue: O / l -> bf16 -> out; each thread owns kColsPerThread of the 128 output columns of its row
         for (int t = 0; t < n_active; ++t) {
@@ -487,8 +428,6 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             if (ok) ok = mbar_wait(smem_u32(&bar->o_full[t]), (n_tiles - 1) & 1, ctl);
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
-            if (tid == 0) TRACE_CTA(6 + t);
-            const int n = q0 + t * kTile + row;
             const uint32_t t_O = lane_base + 256 + t * 128 + part * kColsPerThread;
             if (partial && part == 0)
                 p.part_ml[(size_t)piece_cta * 2 * kTile + t * kTile + row] = make_float2(m_ref[t], l_row);
@@ -538,7 +477,6 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     }
 
     // ---------------------------------------------------------------- tear-down
-    if (tid == 0) TRACE_CTA(8);
     __syncwarp();  // lanes that left a single-lane role loop rejoin before the warp-wide instructions below
     tc_fence_before();
     __syncthreads();
@@ -551,15 +489,9 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         }
         __syncwarp();
         tmem_dealloc(tmem_base, 512);
-        if (lane == 0) TRACE_CTA(9);
     }
 }
 
-#ifdef REGENVC_TRACE
-extern "C" int regenvc_debug_read_trace(long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(g_trace));
-}
-#endif
 
 cudaError_t configure_attn_pipelined() {
     cudaFuncAttributes attr;
