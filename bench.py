@@ -37,8 +37,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 PAPER_CONTEXT = ("paper: 972 ms per 25-frame window (24 fps) for the WHOLE decoder on 8 consumer-class GPUs; "
                  "it reports no attention-only number")
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the self-attention kernel at the 480x832 window
-# shape, from the ncu capture summarised in profiles/attn_pipelined_kernel_window_480x832.md (101.5 MB + 19.1 MB).
-ATTN_KERNEL_DRAM_TRAFFIC_BYTES = {"window_480x832": 120.6e6}
+# shape, from the ncu capture summarised in profiles/attn_pipelined_kernel_window_480x832.md (101.5 MB + 18.0 MB).
+ATTN_KERNEL_DRAM_TRAFFIC_BYTES = {"window_480x832": 119.4e6}
 N_BUFFER_SETS = 4
 
 
