@@ -178,6 +178,22 @@ def test_dominating_key_and_large_scores():
     assert_parity(gpu, ref, float(v.float().abs().max()), "peaked softmax")
 
 
+@pytest.mark.parametrize("growth", [3.0, 12.0, 40.0])
+def test_scores_that_grow_along_the_sequence_force_reference_updates(growth):
+    """Later key tiles hold much larger scores than the first one: the reference set on the first tile must be
+    raised on the way (probabilities would leave the fp16 range otherwise), the accumulator rescaled and the
+    tile redone (several times along the sequence for the larger growth factors)."""
+    T, H, W, h = 1, 24, 50, 2
+    N = T * H * W
+    rng = np.random.default_rng(36)
+    q, v = _rand(rng, N, h, 1.5), _rand(rng, N, h)
+    ramp = (1.0 + (growth - 1.0) * np.arange(N) / (N - 1))[:, None, None]
+    k = synth.from_f32(rng.standard_normal((N, h, D)) * ramp)
+    gpu = f64(run_gpu_self(q, k, v, T, H, W))
+    ref = oracle.self_attention(synth.bits(q), synth.bits(k), synth.bits(v), T, H, W)
+    assert_parity(gpu, ref, float(v.float().abs().max()), f"growing scores x{growth}")
+
+
 def test_heads_are_independent_on_the_gpu():
     T, H, W, h = 2, 9, 10, 4
     N = T * H * W
