@@ -1,26 +1,27 @@
 // Pipelined, warp-specialised tcgen05 attention kernel for sm_100a.
 //
-// One CTA owns one head and two 128-row query tiles (256 query rows):
-//   warps 0-7  softmax: warp w works on TMEM lanes (query rows) 32*(w%4).. and on key columns
-//              64*(w/4)..+63 of every score tile, so two threads share a row; the eight warps take the
-//              score tiles of the two query tiles in turn (S0(j), S1(j), S0(j+1), ...)
-//   warp  8    UMMA issuer (one elected lane) and TMEM owner
-//   warp  9    TMA producer (one elected lane): streams K' and V't tiles
-//   warps 10-11 idle (they complete the third warpgroup, which hands its registers to the softmax warps)
+// One CTA owns one head, two 128-row query tiles (256 query rows) and a range of key tiles:
+//   warps 0-15 softmax (kSplit = 4): warp w works on TMEM lanes (query rows) 32*(w%4).. and on key columns
+//              32*(w/4)..+31 of every score tile, so four threads share a score row; all sixteen warps take
+//              the score tiles of the two query tiles in turn (S0(j), S1(j), S0(j+1), ...)
+//   warp  16   UMMA issuer (one elect.sync-elected lane) and TMEM owner
+//   warp  17   TMA producer (one elected lane): streams K' and V't tiles into a 4-slot ring
+//   warps 18-19 idle (they complete the control warpgroup, which hands registers to the softmax warps)
+// (kSplit = 2 builds the same kernel with eight softmax warps and two threads per row.)
 // While the softmax warps turn S_t into P_t the tensor core runs the other tile's P.V and next Q.K^T.
 //
 // Tensor memory (512 columns x 128 lanes, fp32 cells):
-//   [0,128) S0  [128,256) S1  [256,384) O0  [384,512) O1.  P_t (fp16, two keys per cell) aliases S_t:
-//   keys 0..63 in columns [0,32), keys 64..127 in columns [64,96) of S_t, i.e. each half-row thread writes
-//   its probabilities over score columns it has already read itself.
-// Shared memory: Q0, Q1 (32 KB each, rotated, fp16, 128B-swizzled K-major blocks), then a ring of kStages
-// 32 KB slots holding K'_0, V't_0, K'_1, ...
+//   [0,128) S0  [128,256) S1  [256,384) O0  [384,512) O1.  P_t (fp16, two keys per cell) aliases S_t: the
+//   probabilities of keys [c, c + 32) go to the first 16 of the score columns [c, c + 32), i.e. each thread
+//   writes its probabilities over score columns it has already read itself.
+// Shared memory: Q0, Q1 (32 KB each, rotated, fp16, 128B-swizzled K-major blocks; reused as the staging buffer
+// of the finished output tile), then a ring of kStages 32 KB slots holding K'_0, V't_0, K'_1, ...
 //
 // Softmax keeps, per row, a reference m (log2 domain) and a row sum l.  m is set from the first tile's row
 // maximum and afterwards only raised when a probability would leave the fp16 range (p = 2^(s - m) > 65504),
-// so the probabilities of a tile are formed directly against the reference of the earlier tiles, chunk by
-// chunk as the scores arrive; the threads of a row exchange one float per tile through shared memory to
-// agree on that, and the rescale of the O accumulator (with a redo of the tile) is rare.
+// so the probabilities of a tile are formed directly against the reference of the earlier tiles as soon as
+// the scores arrive; one named barrier with an OR-reduction per tile lets the warps that share 32 rows agree
+// that nothing saturated, and the rescale of the O accumulator (with a redo of the tile) is rare.
 #include "common.cuh"
 #include "ptx.cuh"
 #include "q_tile.cuh"
@@ -56,7 +57,7 @@ constexpr int kMmaWarp = kSoftmaxThreads / 32, kTmaWarp = kMmaWarp + 1;
 // bit i set: pair i of every eight probability pairs takes the polynomial 2^x instead of the MUFU
 constexpr uint32_t kPolyMask = REGENVC_POLY_MASK;
 constexpr uint32_t kIdesc = umma_idesc_f16_f32acc(128, 128);
-constexpr uint32_t kSmemBytes = (2 + kStages) * kTileBytes + 1024 /*align*/ + 256 /*barriers*/ + 16384 /*row exchange*/;
+constexpr uint32_t kSmemBytes = (2 + kStages) * kTileBytes + 1024 /*align*/ + 256 /*barriers*/ + 8192 /*row exchange*/;
 constexpr uint64_t kWaitLimitNs = 500000000ull;   // 0.5 s per wait
 
 struct Barriers {
@@ -71,9 +72,8 @@ struct Barriers {
 };
 static_assert(sizeof(Barriers) <= 256, "barrier block too large");
 
-// Values the two threads of a row hand each other: [parity][tile][half][row].
+// Values the threads of a row hand each other through shared memory (redo path and epilogue only).
 struct RowExchange {
-    float v[2][2][kTile][kSplit];  // partial tile sums: [parity][tile][row][part]
     float m[2][kTile][kSplit];     // partial tile maxima (redo path): [tile][row][part]
     float l[2][kTile][kSplit];     // row sums at the end: [tile][row][part]
 };
