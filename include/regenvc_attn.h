@@ -85,6 +85,31 @@ int regenvc_cross_attn_forward(const void* q, const void* k, const void* v, void
                                int n_q, int n_kv, int n_heads, int head_dim, void* stream);
 
 /*
+ * Block-wise attention for sequence-parallel use (Sec. 3.5: Ring attention streams key/value blocks around
+ * the devices and combines the per-block results "in an online-softmax fashion"; the result equals
+ * unsharded attention up to reduction order).
+ *
+ * regenvc_attn_partial(): attention of a contiguous range of query tokens against ONE contiguous range of
+ * key/value tokens of the same T x H x W grid, left unnormalised.
+ *   q            : device, bf16 [n_q, n_heads, head_dim], tokens q_token0 .. q_token0 + n_q - 1 of the grid
+ *   k, v         : device, bf16 [n_kv, n_heads, head_dim], tokens kv_token0 .. kv_token0 + n_kv - 1
+ *   o_part       : device, fp32 [n_q, n_heads, head_dim]  = sum_m 2^(s_m c - m_row) v_m over the block
+ *                  (c = log2(e) / sqrt(head_dim), s_m the rotated score)
+ *   ml           : device, float pairs [n_q, n_heads]     = (m_row in log2 units, l_row = sum_m 2^(s_m c - m_row))
+ * Rotary positions are those of the tokens in the whole grid, so blocks computed on different devices merge
+ * exactly.  m_row is a reference at or below the block's row maximum plus 16 (not necessarily the maximum).
+ *
+ * regenvc_attn_merge(): out[n, a, :] = sum_i w_i o_i / sum_i w_i l_i with w_i = 2^(m_i - max_i m_i), rounded to
+ * bf16, for n_parts (1..8) partial results of the same query range.  o_parts / mls are HOST arrays of device
+ * pointers.  Merging the partials of a partition of the key range reproduces regenvc_attn_forward().
+ */
+int regenvc_attn_partial(const void* q, const void* k, const void* v, void* o_part, void* ml,
+                         int T, int H, int W, int q_token0, int n_q, int kv_token0, int n_kv,
+                         int n_heads, int head_dim, float rope_theta, void* stream);
+int regenvc_attn_merge(const void* const* o_parts, const void* const* mls, int n_parts, void* out,
+                       int n_q, int n_heads, int head_dim, void* stream);
+
+/*
  * The same two operations for callers whose tensors live in HOST memory
  * (pinned memory gives asynchronous copies; pageable memory works but is
  * staged by the driver).  The call copies q, k, v to device staging buffers

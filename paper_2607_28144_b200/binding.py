@@ -24,7 +24,7 @@ EXPORTS = [
     "regenvc_cross_attn_forward_host", "regenvc_workspace_bytes", "regenvc_set_workspace",
     "regenvc_device_status", "regenvc_status_string", "regenvc_last_cuda_error", "regenvc_version",
     "regenvc_kernel_launch_count", "regenvc_shutdown", "regenvc_debug_set_phases",
-    "regenvc_cross_attn_forward_static",
+    "regenvc_cross_attn_forward_static", "regenvc_attn_partial", "regenvc_attn_merge",
 ]
 
 _lib = None
@@ -52,6 +52,10 @@ def lib() -> ctypes.CDLL:
     L.regenvc_cross_attn_forward.restype = i32
     L.regenvc_cross_attn_forward_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
     L.regenvc_cross_attn_forward_static.restype = i32
+    L.regenvc_attn_partial.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, f32, vp]
+    L.regenvc_attn_partial.restype = i32
+    L.regenvc_attn_merge.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(vp), i32, vp, i32, i32, i32, vp]
+    L.regenvc_attn_merge.restype = i32
     L.regenvc_attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, vp]
     L.regenvc_attn_forward_host.restype = i32
     L.regenvc_cross_attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
@@ -144,6 +148,39 @@ def regenvc_cross_attn_forward_static(q, k, v, out, stream=None):
         raise ValueError("shape mismatch")
     _check(lib().regenvc_cross_attn_forward_static(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), n_q,
                                                    n_kv, h, d, _stream(stream)))
+    return out
+
+
+def regenvc_attn_partial(q, k, v, o_part, ml, T: int, H: int, W: int, q_token0: int, kv_token0: int,
+                         rope_theta: float = 10000.0, stream=None):
+    """Unnormalised attention of the query tokens q_token0.. against the key/value block kv_token0.. of the grid.
+    o_part: CUDA fp32 [n_q, h, d]; ml: CUDA fp32 [n_q, h, 2] (reference, row sum)."""
+    for t, nm in ((q, "q"), (k, "k"), (v, "v")):
+        _dev_bf16(t, nm)
+    n_q, h, d = q.shape
+    n_kv = k.shape[0]
+    if k.shape != (n_kv, h, d) or v.shape != k.shape:
+        raise ValueError("shape mismatch")
+    if o_part.dtype != torch.float32 or tuple(o_part.shape) != (n_q, h, d) or not o_part.is_contiguous():
+        raise TypeError("o_part must be a contiguous CUDA fp32 tensor [n_q, heads, head_dim]")
+    if ml.dtype != torch.float32 or tuple(ml.shape) != (n_q, h, 2) or not ml.is_contiguous():
+        raise TypeError("ml must be a contiguous CUDA fp32 tensor [n_q, heads, 2]")
+    _check(lib().regenvc_attn_partial(q.data_ptr(), k.data_ptr(), v.data_ptr(), o_part.data_ptr(), ml.data_ptr(),
+                                      T, H, W, q_token0, n_q, kv_token0, n_kv, h, d, float(rope_theta),
+                                      _stream(stream)))
+    return o_part, ml
+
+
+def regenvc_attn_merge(o_parts, mls, out, stream=None):
+    """Merges partial results of several key/value blocks (same query range) into bf16 ``out`` [n_q, h, d]."""
+    _dev_bf16(out, "out")
+    n_q, h, d = out.shape
+    n = len(o_parts)
+    if n != len(mls):
+        raise ValueError("need one (m, l) tensor per partial result")
+    arr_o = (ctypes.c_void_p * n)(*[t.data_ptr() for t in o_parts])
+    arr_m = (ctypes.c_void_p * n)(*[t.data_ptr() for t in mls])
+    _check(lib().regenvc_attn_merge(arr_o, arr_m, n, out.data_ptr(), n_q, h, d, _stream(stream)))
     return out
 
 

@@ -199,8 +199,16 @@ size_t operand_bytes(long long n_kv, int n_heads) {
 size_t workspace_need(long long n_kv, int n_heads) { return operand_bytes(n_kv, n_heads) + kSplitScratchBytes; }
 
 // Enqueues the two kernels.  Arguments are already validated; pointers are device pointers.
+// Block-wise use: q and k/v are contiguous token ranges of the T x H x W grid starting at these tokens, and the
+// unnormalised result goes to token-major fp32 buffers instead of `out`.
+struct BlockArgs {
+    int q_token0 = 0, kv_token0 = 0;
+    float* tok_o = nullptr;
+    float2* tok_ml = nullptr;
+};
+
 int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int n_kv, int n_heads, bool rope, int T,
-            int H, int W, float theta, cudaStream_t stream) {
+            int H, int W, float theta, cudaStream_t stream, const BlockArgs& blk = BlockArgs()) {
     std::lock_guard<std::mutex> lock(g_mu);
     int dev = 0;
     DeviceState* st = nullptr;
@@ -244,6 +252,7 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     pp.h = n_heads;
     pp.rope = rope ? 1 : 0;
     pp.grid = grid;
+    pp.pos_offset = blk.kv_token0;
     pp.status = st->status;
     if (tl_phases & 1) {
         CUDA_TRY(launch_prep_kv(pp, stream));
@@ -260,6 +269,9 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     ap.h = n_heads;
     ap.rope = rope ? 1 : 0;
     ap.grid = grid;
+    ap.q_pos_offset = blk.q_token0;
+    ap.tok_o = blk.tok_o;
+    ap.tok_ml = blk.tok_ml;
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)kHeadDim));
     ap.status = st->status;
     ap.sm_count = st->sm_count;
@@ -274,7 +286,7 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     ap.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + operand_bytes(n_kv, n_heads));
     ap.part_ml = reinterpret_cast<float2*>(ap.part_o + (size_t)kMaxPieceCtas * 2 * kTile * kHeadDim);
     const int rem = n_items % st->sm_count;
-    if (rem > 0 && st->sm_count <= kMaxPieceCtas && !split_disabled()) {
+    if (rem > 0 && st->sm_count <= kMaxPieceCtas && !split_disabled() && blk.tok_o == nullptr) {
         int k = st->sm_count / rem;
         if (k > 8) k = 8;
         if (k > n_tiles / 4) k = n_tiles / 4;
@@ -291,7 +303,7 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     }
     // out seen as [n_q rows][n_heads * 128 columns] bf16 for the tiled stores of finished query tiles
     CUtensorMap tmap_out;
-    rc = make_tmap(&tmap_out, out, (uint64_t)n_heads * kHeadDim, (uint64_t)n_q,
+    rc = make_tmap(&tmap_out, out != nullptr ? out : const_cast<void*>(q), (uint64_t)n_heads * kHeadDim, (uint64_t)n_q,
                    (uint64_t)n_heads * kHeadDim * sizeof(__nv_bfloat16), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     if (rc != REGENVC_OK) return rc;
     CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, ap, stream));
@@ -392,6 +404,66 @@ int regenvc_cross_attn_forward_host(const void* q, const void* k, const void* v,
     int rc = validate(q, k, v, out, n_q, n_kv, n_heads, head_dim, false);
     if (rc != REGENVC_OK) return rc;
     return run_host(q, k, v, out, n_q, n_kv, n_heads, false, 1, 1, 1, 1.0f, (cudaStream_t)stream);
+}
+
+int regenvc_attn_partial(const void* q, const void* k, const void* v, void* o_part, void* ml, int T, int H, int W,
+                         int q_token0, int n_q, int kv_token0, int n_kv, int n_heads, int head_dim, float rope_theta,
+                         void* stream) {
+    if (!q || !k || !v || !o_part || !ml) return REGENVC_ERR_NULL_POINTER;
+    long long n = 0;
+    int rc = check_self_args(T, H, W, rope_theta, &n);
+    if (rc != REGENVC_OK) return rc;
+    if (q_token0 < 0 || kv_token0 < 0 || n_q < 1 || n_kv < 1 || (long long)q_token0 + n_q > n ||
+        (long long)kv_token0 + n_kv > n)
+        return REGENVC_ERR_BAD_SHAPE;
+    // the ordinary checks, with o_part standing in for out (it is larger, so an overlap test on it is stricter)
+    rc = validate(q, k, v, o_part, n_q, n_kv, n_heads, head_dim, true);
+    if (rc != REGENVC_OK) return rc;
+    if (((uintptr_t)ml) & 15) return REGENVC_ERR_MISALIGNED;
+    const size_t qb = (size_t)n_q * n_heads * head_dim * 2, kb = (size_t)n_kv * n_heads * head_dim * 2;
+    const size_t ob = 2 * qb, mb = (size_t)n_q * n_heads * sizeof(float2);
+    if (overlaps(o_part, ob, q, qb) || overlaps(o_part, ob, k, kb) || overlaps(o_part, ob, v, kb) ||
+        overlaps(ml, mb, q, qb) || overlaps(ml, mb, k, kb) || overlaps(ml, mb, v, kb) || overlaps(ml, mb, o_part, ob))
+        return REGENVC_ERR_ALIASING;
+    if (!(rope_theta > 0.0f) || !std::isfinite(rope_theta)) return REGENVC_ERR_UNSUPPORTED;
+    BlockArgs blk;
+    blk.q_token0 = q_token0;
+    blk.kv_token0 = kv_token0;
+    blk.tok_o = reinterpret_cast<float*>(o_part);
+    blk.tok_ml = reinterpret_cast<float2*>(ml);
+    return enqueue(q, k, v, nullptr, n_q, n_kv, n_heads, true, T, H, W, rope_theta, (cudaStream_t)stream, blk);
+}
+
+int regenvc_attn_merge(const void* const* o_parts, const void* const* mls, int n_parts, void* out, int n_q,
+                       int n_heads, int head_dim, void* stream) {
+    if (!o_parts || !mls || !out) return REGENVC_ERR_NULL_POINTER;
+    if (n_parts < 1 || n_parts > kMaxMergeParts || n_q < 1 || n_heads < 1) return REGENVC_ERR_BAD_SHAPE;
+    if (head_dim != kHeadDim) return REGENVC_ERR_UNSUPPORTED;
+    TokenMergeParams mp;
+    const size_t rows = (size_t)n_q * n_heads;
+    for (int i = 0; i < n_parts; ++i) {
+        if (!o_parts[i] || !mls[i]) return REGENVC_ERR_NULL_POINTER;
+        if ((((uintptr_t)o_parts[i]) | ((uintptr_t)mls[i])) & 15) return REGENVC_ERR_MISALIGNED;
+        if (overlaps(out, rows * kHeadDim * 2, o_parts[i], rows * kHeadDim * 4) ||
+            overlaps(out, rows * kHeadDim * 2, mls[i], rows * sizeof(float2)))
+            return REGENVC_ERR_ALIASING;
+        mp.o[i] = reinterpret_cast<const float*>(o_parts[i]);
+        mp.ml[i] = reinterpret_cast<const float2*>(mls[i]);
+    }
+    if (((uintptr_t)out) & 15) return REGENVC_ERR_MISALIGNED;
+    mp.n_parts = n_parts;
+    mp.out = reinterpret_cast<__nv_bfloat16*>(out);
+    mp.n_rows = (long long)rows;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        int dev = 0;
+        DeviceState* st = nullptr;
+        int rc = device_state(&dev, &st);
+        if (rc != REGENVC_OK) return rc;
+    }
+    CUDA_TRY(launch_merge_token_partials(mp, (cudaStream_t)stream));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return REGENVC_OK;
 }
 
 size_t regenvc_workspace_bytes(int n_kv, int n_heads, int head_dim) {

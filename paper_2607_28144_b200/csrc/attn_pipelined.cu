@@ -187,9 +187,10 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     // work item and key-tile range of this CTA
     const int n_tiles_total = p.n_kv_pad / kTile;
     int item = blockIdx.x, kv_tile0 = 0, n_tiles = n_tiles_total;
-    const bool partial = static_cast<int>(blockIdx.x) >= p.n_full_items;
+    const bool piece = static_cast<int>(blockIdx.x) >= p.n_full_items;  // one of several key-range pieces of an item
+    const bool partial = piece || p.tok_o != nullptr;                     // leaves an unnormalised result
     const int piece_cta = static_cast<int>(blockIdx.x) - p.n_full_items;
-    if (partial) {
+    if (piece) {
         item = p.n_full_items + piece_cta / p.split_k;
         kv_tile0 = (piece_cta % p.split_k) * p.tiles_per_piece;
         n_tiles = min(p.tiles_per_piece, n_tiles_total - kv_tile0);
@@ -429,8 +430,11 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
             const uint32_t t_O = lane_base + 256 + t * 128 + part * kColsPerThread;
-            if (partial && part == 0)
-                p.part_ml[(size_t)piece_cta * 2 * kTile + t * kTile + row] = make_float2(m_ref[t], l_row);
+            const int n_row = q0 + t * kTile + row;  // query row of this thread
+            if (partial && part == 0) {
+                if (piece) p.part_ml[(size_t)piece_cta * 2 * kTile + t * kTile + row] = make_float2(m_ref[t], l_row);
+                else if (n_row < p.n_q) p.tok_ml[(size_t)n_row * p.h + head] = make_float2(m_ref[t], l_row);
+            }
 #pragma unroll 1
             for (int cb = 0; cb < kChunks; ++cb) {
                 uint32_t o[32];
@@ -439,11 +443,14 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     tmem_wait_ld();
                 }
                 if (ok && partial) {
-                    // unnormalised fp32 row part for the merge kernel
-                    uint4* dst = reinterpret_cast<uint4*>(p.part_o + ((size_t)piece_cta * 2 * kTile + t * kTile + row) * kHeadDim +
-                                                          part * kColsPerThread + cb * 32);
+                    // unnormalised fp32 row part for a merge kernel: piece scratch, or the caller's token-major buffer
+                    float* row_o = piece ? p.part_o + ((size_t)piece_cta * 2 * kTile + t * kTile + row) * kHeadDim
+                                         : p.tok_o + ((size_t)n_row * p.h + head) * kHeadDim;
+                    uint4* dst = reinterpret_cast<uint4*>(row_o + part * kColsPerThread + cb * 32);
+                    if (piece || n_row < p.n_q) {
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) dst[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                        for (int c = 0; c < 8; ++c) dst[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                    }
                 } else if (ok) {
                     // normalised bf16 row part into the (now idle) query tile buffer, in the swizzled layout of a
                     // TMA box {64 columns, 128 rows}; one tiled store per 64-column block writes the tile out

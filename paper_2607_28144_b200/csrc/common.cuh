@@ -35,6 +35,7 @@ struct PrepParams {
     int n_kv, n_kv_pad, h;
     int rope;                 // 1: rotate k by the 3D rotary embedding
     RopeGrid grid;
+    int pos_offset;           // token index (in the T x H x W grid) of row 0 of k
     int* status;
 };
 
@@ -55,8 +56,23 @@ struct AttnParams {
     int n_full_items;
     int split_k;              // >= 1
     int tiles_per_piece;
+    int q_pos_offset;         // token index (in the T x H x W grid) of row 0 of q
+    // Token-major partial output (block-wise attention for ring-style merging): when tok_o is not null every
+    // CTA leaves its unnormalised result here instead of writing `out`.
+    float* tok_o;             // [n_q, h, 128] fp32, sum_m 2^(s_m c - m_row) v_m
+    float2* tok_ml;           // [n_q, h] (m_row in log2 units, l_row)
     float* part_o;            // [piece CTA][256 rows][128] fp32, sum_m p_m v_m against the piece's reference
     float2* part_ml;          // [piece CTA][256 rows] (reference m in log2 units, row sum l)
+};
+
+// Merge of token-major partial results of several key/value blocks.
+constexpr int kMaxMergeParts = 8;
+struct TokenMergeParams {
+    const float* o[kMaxMergeParts];
+    const float2* ml[kMaxMergeParts];
+    int n_parts;
+    __nv_bfloat16* out;       // [n_q, h, 128]
+    long long n_rows;         // n_q * h
 };
 
 struct MergeParams {
@@ -73,6 +89,7 @@ cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& 
                                   const AttnParams& p, cudaStream_t stream);
 cudaError_t configure_attn_pipelined();   // once per device: register hand-over check, large dynamic shared memory
 cudaError_t launch_merge_partials(const MergeParams& p, cudaStream_t stream);
+cudaError_t launch_merge_token_partials(const TokenMergeParams& p, cudaStream_t stream);
 
 // Bytes of the partial-result scratch that follows K' and V't in the workspace: room for up to
 // kMaxPieceCtas piece CTAs (never more than one wave of SMs is cut into pieces).

@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
             const int n = tile0 + it * 16 + (tid >> 4);
             float x[8];
             bf16x8_to_float(raw[it], x);
-            if (p.rope && n < p.n_kv) rope_rotate8(x, p.grid, token_pos(n, p.grid), chunk);
+            if (p.rope && n < p.n_kv) rope_rotate8(x, p.grid, token_pos(n + p.pos_offset, p.grid), chunk);
 #pragma unroll
             for (int i = 0; i < 8; ++i) out_of_range |= !(fabsf(x[i]) <= 65504.0f);
             uint4 packed;

@@ -38,7 +38,7 @@ __device__ __forceinline__ void load_rotate_q_tiles(const AttnParams& p, int hea
             const int n = q0 + t * kTile + row;
             float x[8];
             bf16x8_to_float(raw[t][it], x);
-            if (p.rope && n < p.n_q) rope_rotate8(x, p.grid, token_pos(n, p.grid), chunk);
+            if (p.rope && n < p.n_q) rope_rotate8(x, p.grid, token_pos(n + p.q_pos_offset, p.grid), chunk);
             uint4 packed;
             packed.x = pack_f16x2(x[0], x[1]);
             packed.y = pack_f16x2(x[2], x[3]);

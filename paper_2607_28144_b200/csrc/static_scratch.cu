@@ -122,6 +122,7 @@ extern "C" int regenvc_cross_attn_forward_static(const void* q, const void* k, c
     pp.h = n_heads;
     pp.rope = 0;
     pp.grid = RopeGrid{nullptr, 1, 1, 1};
+    pp.pos_offset = 0;
     pp.status = dev->status;
     if (launch_prep_kv(pp, (cudaStream_t)stream) != cudaSuccess) return REGENVC_ERR_CUDA;
 
@@ -141,6 +142,9 @@ extern "C" int regenvc_cross_attn_forward_static(const void* q, const void* k, c
     ap.n_full_items = ap.pairs_per_head * n_heads;  // no key-range pieces: they would need more scratch
     ap.split_k = 1;
     ap.tiles_per_piece = (int)(kv_pad / kTile);
+    ap.q_pos_offset = 0;
+    ap.tok_o = nullptr;
+    ap.tok_ml = nullptr;
     ap.part_o = nullptr;
     ap.part_ml = nullptr;
     if (launch_attn_pipelined(tmap_k, tmap_v, tmap_out, ap, (cudaStream_t)stream) != cudaSuccess) return REGENVC_ERR_CUDA;
