@@ -114,7 +114,13 @@ int regenvc_attn_merge(const void* const* o_parts, const void* const* mls, int n
  * (pinned memory gives asynchronous copies; pageable memory works but is
  * staged by the driver).  The call copies q, k, v to device staging buffers
  * that the library owns and reuses, runs the device path, copies the result
- * back into `out` and waits for `stream` before returning.
+ * back into `out` and waits for `stream` before returning.  K and V are
+ * copied first; the query rows follow in up to 8 blocks of at least one wave
+ * of work items, and the library's own copy-in and copy-out streams overlap
+ * the transfer of a block with the attention of the previous one (all of it
+ * ordered after the work already on `stream`).  The result equals the device
+ * call's to the last bf16 step: a block is cut into work items of its own, so
+ * a row can see another rounding of its fp16 probabilities.
  */
 int regenvc_attn_forward_host(const void* q, const void* k, const void* v, void* out,
                               int T, int H, int W, int n_heads, int head_dim,

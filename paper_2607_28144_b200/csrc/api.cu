@@ -32,6 +32,15 @@ struct RopeEntry {
     float theta;
     float2* dev;
 };
+// Streams and events of the host-buffer entry points: copies in, kernels and copies out run on three streams
+// so that the transfer of one block of query rows overlaps the attention of the previous one.
+constexpr int kMaxHostChunks = 8;
+struct HostPipe {
+    bool made = false;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, kv = nullptr, fin = nullptr;
+    cudaEvent_t q[kMaxHostChunks] = {}, done[kMaxHostChunks] = {};
+};
 struct DeviceState {
     bool checked = false, supported = false;
     int* status = nullptr;
@@ -39,6 +48,7 @@ struct DeviceState {
     std::vector<RopeEntry> ropes;
     std::map<std::thread::id, Buf> workspace;
     std::map<std::thread::id, std::vector<Buf>> staging;  // q, k, v, out
+    std::map<std::thread::id, HostPipe> pipes;
 };
 
 std::mutex g_mu;
@@ -205,6 +215,7 @@ struct BlockArgs {
     int q_token0 = 0, kv_token0 = 0;
     float* tok_o = nullptr;
     float2* tok_ml = nullptr;
+    int phases = -1;  // bit 0: preparation pass, bit 1: attention; -1: the calling thread's debug setting
 };
 
 int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int n_kv, int n_heads, bool rope, int T,
@@ -254,11 +265,12 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     pp.grid = grid;
     pp.pos_offset = blk.kv_token0;
     pp.status = st->status;
-    if (tl_phases & 1) {
+    const int phases = blk.phases >= 0 ? blk.phases : tl_phases;
+    if (phases & 1) {
         CUDA_TRY(launch_prep_kv(pp, stream));
         g_launches.fetch_add(1, std::memory_order_relaxed);
     }
-    if (!(tl_phases & 2)) return REGENVC_OK;
+    if (!(phases & 2)) return REGENVC_OK;
 
     AttnParams ap;
     ap.q = reinterpret_cast<const __nv_bfloat16*>(q);
@@ -325,11 +337,32 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     return REGENVC_OK;
 }
 
-// Host-buffer variant: stage in, run, stage out, wait.
+int make_pipe(HostPipe& hp) {
+    if (hp.made) return REGENVC_OK;
+    CUDA_TRY(cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking));
+    CUDA_TRY(cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking));
+    CUDA_TRY(cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming));
+    CUDA_TRY(cudaEventCreateWithFlags(&hp.kv, cudaEventDisableTiming));
+    CUDA_TRY(cudaEventCreateWithFlags(&hp.fin, cudaEventDisableTiming));
+    for (int c = 0; c < kMaxHostChunks; ++c) {
+        CUDA_TRY(cudaEventCreateWithFlags(&hp.q[c], cudaEventDisableTiming));
+        CUDA_TRY(cudaEventCreateWithFlags(&hp.done[c], cudaEventDisableTiming));
+    }
+    hp.made = true;
+    return REGENVC_OK;
+}
+
+// Host-buffer variant: stage in, run, stage out, wait.  K and V go first (the preparation pass needs them whole);
+// the query rows follow in blocks of whole waves of work items, and each block's attention and the copy of its
+// result back overlap the transfer of the next block.
 int run_host(const void* q, const void* k, const void* v, void* out, int n_q, int n_kv, int n_heads, bool rope, int T,
              int H, int W, float theta, cudaStream_t stream) {
-    const size_t qb = (size_t)n_q * n_heads * kHeadDim * 2, kb = (size_t)n_kv * n_heads * kHeadDim * 2;
-    void *dq, *dk, *dv, *dout;
+    const size_t row_bytes = (size_t)n_heads * kHeadDim * 2;
+    const size_t qb = (size_t)n_q * row_bytes, kb = (size_t)n_kv * row_bytes;
+    char *dq, *dout;
+    void *dk, *dv;
+    HostPipe* hp = nullptr;
+    int sm_count = 1;
     {
         std::lock_guard<std::mutex> lock(g_mu);
         int dev = 0;
@@ -343,14 +376,50 @@ int run_host(const void* q, const void* k, const void* v, void* out, int n_q, in
             rc = grow(s[i], need[i]);
             if (rc != REGENVC_OK) return rc;
         }
-        dq = s[0].ptr; dk = s[1].ptr; dv = s[2].ptr; dout = s[3].ptr;
+        dq = (char*)s[0].ptr; dk = s[1].ptr; dv = s[2].ptr; dout = (char*)s[3].ptr;
+        hp = &st->pipes[std::this_thread::get_id()];
+        rc = make_pipe(*hp);
+        if (rc != REGENVC_OK) return rc;
+        sm_count = st->sm_count > 0 ? st->sm_count : 1;
     }
-    CUDA_TRY(cudaMemcpyAsync(dq, q, qb, cudaMemcpyHostToDevice, stream));
-    CUDA_TRY(cudaMemcpyAsync(dk, k, kb, cudaMemcpyHostToDevice, stream));
-    CUDA_TRY(cudaMemcpyAsync(dv, v, kb, cudaMemcpyHostToDevice, stream));
-    int rc = enqueue(dq, dk, dv, dout, n_q, n_kv, n_heads, rope, T, H, W, theta, stream);
+    // blocks of query rows: at least one full wave of (head x 256 rows) work items each, at most kMaxHostChunks
+    const int pairs = (n_q + 2 * kTile - 1) / (2 * kTile);
+    int n_chunks = (int)(((long long)pairs * n_heads) / sm_count);
+    if (n_chunks < 1) n_chunks = 1;
+    if (n_chunks > kMaxHostChunks) n_chunks = kMaxHostChunks;
+    if (n_chunks > pairs) n_chunks = pairs;
+    const int rows_per_chunk = (pairs + n_chunks - 1) / n_chunks * 2 * kTile;
+
+    // the copies start after whatever the caller has already put on its stream
+    CUDA_TRY(cudaEventRecord(hp->start, stream));
+    CUDA_TRY(cudaStreamWaitEvent(hp->in, hp->start, 0));
+    CUDA_TRY(cudaStreamWaitEvent(hp->out, hp->start, 0));
+    CUDA_TRY(cudaMemcpyAsync(dk, k, kb, cudaMemcpyHostToDevice, hp->in));
+    CUDA_TRY(cudaMemcpyAsync(dv, v, kb, cudaMemcpyHostToDevice, hp->in));
+    CUDA_TRY(cudaEventRecord(hp->kv, hp->in));
+    CUDA_TRY(cudaStreamWaitEvent(stream, hp->kv, 0));
+    BlockArgs prep;
+    prep.phases = 1;
+    int rc = enqueue(dq, dk, dv, dout, n_q, n_kv, n_heads, rope, T, H, W, theta, stream, prep);
     if (rc != REGENVC_OK) return rc;
-    CUDA_TRY(cudaMemcpyAsync(out, dout, qb, cudaMemcpyDeviceToHost, stream));
+    int c = 0;
+    for (int r0 = 0; r0 < n_q; r0 += rows_per_chunk, ++c) {
+        const int rows = n_q - r0 < rows_per_chunk ? n_q - r0 : rows_per_chunk;
+        const size_t off = (size_t)r0 * row_bytes, bytes = (size_t)rows * row_bytes;
+        CUDA_TRY(cudaMemcpyAsync(dq + off, (const char*)q + off, bytes, cudaMemcpyHostToDevice, hp->in));
+        CUDA_TRY(cudaEventRecord(hp->q[c], hp->in));
+        CUDA_TRY(cudaStreamWaitEvent(stream, hp->q[c], 0));
+        BlockArgs blk;
+        blk.phases = 2;
+        blk.q_token0 = r0;
+        rc = enqueue(dq + off, dk, dv, dout + off, rows, n_kv, n_heads, rope, T, H, W, theta, stream, blk);
+        if (rc != REGENVC_OK) return rc;
+        CUDA_TRY(cudaEventRecord(hp->done[c], stream));
+        CUDA_TRY(cudaStreamWaitEvent(hp->out, hp->done[c], 0));
+        CUDA_TRY(cudaMemcpyAsync((char*)out + off, dout + off, bytes, cudaMemcpyDeviceToHost, hp->out));
+    }
+    CUDA_TRY(cudaEventRecord(hp->fin, hp->out));
+    CUDA_TRY(cudaStreamWaitEvent(stream, hp->fin, 0));
     CUDA_TRY(cudaStreamSynchronize(stream));
     return REGENVC_OK;
 }
@@ -542,6 +611,19 @@ void regenvc_shutdown(void) {
         for (auto& w : st.workspace) cudaFree(w.second.ptr);
         for (auto& s : st.staging)
             for (Buf& b : s.second) cudaFree(b.ptr);
+        for (auto& hp : st.pipes) {
+            HostPipe& h = hp.second;
+            if (!h.made) continue;
+            cudaStreamDestroy(h.in);
+            cudaStreamDestroy(h.out);
+            cudaEventDestroy(h.start);
+            cudaEventDestroy(h.kv);
+            cudaEventDestroy(h.fin);
+            for (int c = 0; c < kMaxHostChunks; ++c) {
+                cudaEventDestroy(h.q[c]);
+                cudaEventDestroy(h.done[c]);
+            }
+        }
     }
     g_dev.clear();
     cudaSetDevice(prev);
