@@ -110,6 +110,32 @@ int regenvc_attn_merge(const void* const* o_parts, const void* const* mls, int n
                        int n_q, int n_heads, int head_dim, void* stream);
 
 /*
+ * Head <-> sequence resharding of the Ulysses scheme (Sec. 3.5: an all-to-all moves the sequence sharding
+ * into the head dimension before attention and back afterwards, so that each GPU attends over the whole
+ * sequence for a subset of the heads).  These two calls are the data movement of that all-to-all for one
+ * GPU of a group of `world` (1..16) GPUs; all tensors are bf16 with head_dim = 128, device pointers, 16-byte
+ * aligned.  `dst` is a HOST array of `world` device pointers.  A destination may be memory of this GPU (a
+ * send buffer that a collective ships afterwards) or a peer GPU's buffer mapped into this process: then the
+ * stores cross NVLink and the call is the exchange itself.  The library only writes; ordering between GPUs
+ * (nobody reads a buffer before all writers have finished, nobody overwrites one that is still being read)
+ * is the caller's, by stream events or a barrier.  Asynchronous on `stream`; no allocation.
+ *
+ * regenvc_ulysses_scatter_heads(): x_local is this GPU's token range [n_local, n_heads, 128].  For every
+ *   r < world: dst[r][dst_token0 + n, a, :] = x_local[n, r * n_heads / world + a, :], dst[r] laid out
+ *   [tokens of the group, n_heads / world, 128].  n_heads must be a multiple of world.
+ * regenvc_ulysses_gather_heads(): x_heads is this GPU's head range of all tokens of the group
+ *   [*, n_heads_local, 128].  For every r < world: dst[r][n, dst_head0 + a, :] = x_heads[token0[r] + n, a, :]
+ *   for n < n_tokens[r], dst[r] laid out [n_tokens[r], n_heads_dst, 128].  token0 / n_tokens are HOST arrays.
+ * Errors: NULL_POINTER, BAD_SHAPE (world, head counts, negative sizes, 32-bit row index overflow),
+ * UNSUPPORTED (head_dim), MISALIGNED, ALIASING (a destination range overlaps the source), CUDA.
+ */
+int regenvc_ulysses_scatter_heads(const void* x_local, void* const* dst, int world, int n_local,
+                                  int dst_token0, int n_heads, int head_dim, void* stream);
+int regenvc_ulysses_gather_heads(const void* x_heads, void* const* dst, const int* token0,
+                                 const int* n_tokens, int world, int n_heads_local, int n_heads_dst,
+                                 int dst_head0, int head_dim, void* stream);
+
+/*
  * The same two operations for callers whose tensors live in HOST memory
  * (pinned memory gives asynchronous copies; pageable memory works but is
  * staged by the driver).  The call copies q, k, v to device staging buffers

@@ -25,6 +25,7 @@ EXPORTS = [
     "regenvc_device_status", "regenvc_status_string", "regenvc_last_cuda_error", "regenvc_version",
     "regenvc_kernel_launch_count", "regenvc_shutdown", "regenvc_debug_set_phases",
     "regenvc_cross_attn_forward_static", "regenvc_attn_partial", "regenvc_attn_merge",
+    "regenvc_ulysses_scatter_heads", "regenvc_ulysses_gather_heads",
 ]
 
 _lib = None
@@ -56,6 +57,11 @@ def lib() -> ctypes.CDLL:
     L.regenvc_attn_partial.restype = i32
     L.regenvc_attn_merge.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(vp), i32, vp, i32, i32, i32, vp]
     L.regenvc_attn_merge.restype = i32
+    L.regenvc_ulysses_scatter_heads.argtypes = [vp, ctypes.POINTER(vp), i32, i32, i32, i32, i32, vp]
+    L.regenvc_ulysses_scatter_heads.restype = i32
+    L.regenvc_ulysses_gather_heads.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                               i32, i32, i32, i32, i32, vp]
+    L.regenvc_ulysses_gather_heads.restype = i32
     L.regenvc_attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, vp]
     L.regenvc_attn_forward_host.restype = i32
     L.regenvc_cross_attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
@@ -182,6 +188,38 @@ def regenvc_attn_merge(o_parts, mls, out, stream=None):
     arr_m = (ctypes.c_void_p * n)(*[t.data_ptr() for t in mls])
     _check(lib().regenvc_attn_merge(arr_o, arr_m, n, out.data_ptr(), n_q, h, d, _stream(stream)))
     return out
+
+
+def _ptr(x) -> int:
+    return x.data_ptr() if isinstance(x, torch.Tensor) else int(x)
+
+
+def regenvc_ulysses_scatter_heads(x_local, dst, dst_token0: int, stream=None):
+    """Head-group r of this GPU's tokens ``x_local`` [n_local, h, d] goes to ``dst[r]`` [group tokens, h/len(dst), d]
+    at rows ``dst_token0``...  ``dst`` holds CUDA tensors or raw device addresses (a peer GPU's mapped buffer)."""
+    _dev_bf16(x_local, "x_local")
+    n, h, d = x_local.shape
+    world = len(dst)
+    arr = (ctypes.c_void_p * world)(*[_ptr(t) for t in dst])
+    _check(lib().regenvc_ulysses_scatter_heads(x_local.data_ptr(), arr, world, n, int(dst_token0), h, d,
+                                               _stream(stream)))
+
+
+def regenvc_ulysses_gather_heads(x_heads, dst, token0, n_tokens, n_heads_dst: int, dst_head0: int, stream=None):
+    """Tokens ``token0[r]``.. (``n_tokens[r]`` of them) of this GPU's heads ``x_heads`` [tokens, h_local, d] go to
+    ``dst[r]`` [n_tokens[r], n_heads_dst, d] at heads ``dst_head0``...  ``dst`` as in the scatter call."""
+    _dev_bf16(x_heads, "x_heads")
+    _, h_loc, d = x_heads.shape
+    world = len(dst)
+    if len(token0) != world or len(n_tokens) != world:
+        raise ValueError("need one token range per destination")
+    if any(t0 < 0 or n < 0 or t0 + n > x_heads.shape[0] for t0, n in zip(token0, n_tokens)):
+        raise ValueError("token range outside x_heads")
+    arr = (ctypes.c_void_p * world)(*[_ptr(t) for t in dst])
+    a0 = (ctypes.c_int * world)(*[int(x) for x in token0])
+    an = (ctypes.c_int * world)(*[int(x) for x in n_tokens])
+    _check(lib().regenvc_ulysses_gather_heads(x_heads.data_ptr(), arr, a0, an, world, h_loc, int(n_heads_dst),
+                                              int(dst_head0), d, _stream(stream)))
 
 
 def regenvc_attn_forward_host(q, k, v, out, T: int, H: int, W: int, rope_theta: float = 10000.0, stream=None):

@@ -535,6 +535,92 @@ int regenvc_attn_merge(const void* const* o_parts, const void* const* mls, int n
     return REGENVC_OK;
 }
 
+int regenvc_ulysses_scatter_heads(const void* x_local, void* const* dst, int world, int n_local, int dst_token0,
+                                  int n_heads, int head_dim, void* stream) {
+    if (!x_local || !dst) return REGENVC_ERR_NULL_POINTER;
+    if (world < 1 || world > kMaxReshardPeers || n_local < 0 || dst_token0 < 0 || n_heads < 1 || n_heads % world != 0)
+        return REGENVC_ERR_BAD_SHAPE;
+    if ((long long)(dst_token0 + (long long)n_local) * n_heads >= (1ll << 31)) return REGENVC_ERR_BAD_SHAPE;
+    if (head_dim != kHeadDim) return REGENVC_ERR_UNSUPPORTED;
+    if ((uintptr_t)x_local & 15) return REGENVC_ERR_MISALIGNED;
+    ReshardParams rp{};
+    rp.src = reinterpret_cast<const uint4*>(x_local);
+    rp.world = world;
+    rp.h_src = n_heads;
+    rp.h_dst = n_heads / world;
+    rp.dst_row0 = dst_token0;
+    rp.dst_head0 = 0;
+    const size_t src_bytes = (size_t)n_local * n_heads * kHeadDim * 2;
+    for (int r = 0; r < world; ++r) {
+        if (!dst[r]) return REGENVC_ERR_NULL_POINTER;
+        if ((uintptr_t)dst[r] & 15) return REGENVC_ERR_MISALIGNED;
+        const char* first = (const char*)dst[r] + (size_t)dst_token0 * rp.h_dst * kHeadDim * 2;
+        if (overlaps(first, src_bytes / world, x_local, src_bytes)) return REGENVC_ERR_ALIASING;
+        rp.dst[r] = reinterpret_cast<uint4*>(dst[r]);
+        rp.row0[r] = 0;
+        rp.rows[r] = n_local;
+    }
+    int sm_count = 0;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        int dev = 0;
+        DeviceState* st = nullptr;
+        int rc = device_state(&dev, &st);
+        if (rc != REGENVC_OK) return rc;
+        sm_count = st->sm_count;
+    }
+    if (n_local == 0) return REGENVC_OK;
+    CUDA_TRY(launch_scatter_heads(rp, sm_count, (cudaStream_t)stream));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return REGENVC_OK;
+}
+
+int regenvc_ulysses_gather_heads(const void* x_heads, void* const* dst, const int* token0, const int* n_tokens,
+                                 int world, int n_heads_local, int n_heads_dst, int dst_head0, int head_dim,
+                                 void* stream) {
+    if (!x_heads || !dst || !token0 || !n_tokens) return REGENVC_ERR_NULL_POINTER;
+    if (world < 1 || world > kMaxReshardPeers || n_heads_local < 1 || n_heads_dst < n_heads_local || dst_head0 < 0 ||
+        dst_head0 + n_heads_local > n_heads_dst)
+        return REGENVC_ERR_BAD_SHAPE;
+    if (head_dim != kHeadDim) return REGENVC_ERR_UNSUPPORTED;
+    if ((uintptr_t)x_heads & 15) return REGENVC_ERR_MISALIGNED;
+    ReshardParams rp{};
+    rp.src = reinterpret_cast<const uint4*>(x_heads);
+    rp.world = world;
+    rp.h_src = n_heads_local;
+    rp.h_dst = n_heads_dst;
+    rp.dst_row0 = 0;
+    rp.dst_head0 = dst_head0;
+    long long total = 0;
+    for (int r = 0; r < world; ++r) {
+        if (!dst[r]) return REGENVC_ERR_NULL_POINTER;
+        if ((uintptr_t)dst[r] & 15) return REGENVC_ERR_MISALIGNED;
+        if (token0[r] < 0 || n_tokens[r] < 0) return REGENVC_ERR_BAD_SHAPE;
+        if (((long long)token0[r] + n_tokens[r]) * n_heads_dst >= (1ll << 31)) return REGENVC_ERR_BAD_SHAPE;
+        const char* from = (const char*)x_heads + (size_t)token0[r] * n_heads_local * kHeadDim * 2;
+        if (overlaps(dst[r], (size_t)n_tokens[r] * n_heads_dst * kHeadDim * 2, from,
+                     (size_t)n_tokens[r] * n_heads_local * kHeadDim * 2))
+            return REGENVC_ERR_ALIASING;
+        rp.dst[r] = reinterpret_cast<uint4*>(dst[r]);
+        rp.row0[r] = token0[r];
+        rp.rows[r] = n_tokens[r];
+        total += n_tokens[r];
+    }
+    int sm_count = 0;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        int dev = 0;
+        DeviceState* st = nullptr;
+        int rc = device_state(&dev, &st);
+        if (rc != REGENVC_OK) return rc;
+        sm_count = st->sm_count;
+    }
+    if (total == 0) return REGENVC_OK;
+    CUDA_TRY(launch_gather_heads(rp, sm_count, (cudaStream_t)stream));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return REGENVC_OK;
+}
+
 size_t regenvc_workspace_bytes(int n_kv, int n_heads, int head_dim) {
     if (n_kv < 1 || n_heads < 1 || head_dim != kHeadDim) return 0;
     return workspace_need(n_kv, n_heads);

@@ -83,6 +83,24 @@ struct MergeParams {
     int pairs_per_head, n_full_items, split_k, n_split_items;
 };
 
+// Head <-> sequence resharding (Ulysses, Sec. 3.5).  Rows are (token, head) vectors of 128 bf16 = 16 uint4.
+//   scatter: src [n_rows][h_src] -> for every destination r: dst[r][(dst_row0 + n)][h_dst] = src[n][r * h_dst + .]
+//   gather : src [.][h_src]      -> for every destination r: dst[r][n][dst_head0 + .] = src[row0[r] + n][.],
+//            n < rows[r], destination rows holding h_dst heads
+constexpr int kMaxReshardPeers = 16;
+struct ReshardParams {
+    const uint4* src;
+    uint4* dst[kMaxReshardPeers];
+    int row0[kMaxReshardPeers];   // gather: first source row of destination r
+    int rows[kMaxReshardPeers];   // rows copied to destination r (scatter: all equal to the source's row count)
+    int world;
+    int h_src, h_dst;
+    int dst_row0;                 // scatter only
+    int dst_head0;                // gather only
+};
+cudaError_t launch_scatter_heads(const ReshardParams& p, int sm_count, cudaStream_t stream);
+cudaError_t launch_gather_heads(const ReshardParams& p, int sm_count, cudaStream_t stream);
+
 // Launchers (each returns the launch error, enqueues on `stream`).
 cudaError_t launch_prep_kv(const PrepParams& p, cudaStream_t stream);
 cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
