@@ -29,7 +29,13 @@
  *     nor keeps them beyond the stream-ordered work of the call.
  *   - Device entry points are asynchronous on `stream` (a cudaStream_t cast
  *     to void*, NULL = legacy default stream) and never synchronise the host
- *     once the workspace and the rotary table for the shape exist.
+ *     once the workspace and the rotary table for the shape exist.  Such a
+ *     warm call only enqueues kernels (their parameters, tensor maps
+ *     included, travel by value), so a sequence of warm calls can be
+ *     recorded into a CUDA graph and replayed on new values in the same
+ *     buffers (regenvc_attn_forward, regenvc_cross_attn_forward,
+ *     regenvc_attn_partial, regenvc_attn_merge, the resharding calls; not
+ *     the *_host variants, which copy and wait).
  *   - Errors are return codes only; arguments are validated before any CUDA
  *     work is enqueued, and a failing call enqueues nothing.
  *   - There is no CPU path: on a machine without an sm_100 GPU every compute

@@ -243,3 +243,37 @@ def test_workspace_too_small_is_rejected():
         assert ei.value.code == binding.ERR_WORKSPACE
     finally:
         binding.regenvc_set_workspace(None)
+
+
+def test_warm_calls_can_be_captured_in_a_cuda_graph_and_replayed():
+    """A warm call allocates nothing and never synchronises, so a whole step (self-attention plus cross-attention)
+    can be recorded once and replayed; the replay on new input values must equal direct calls bit for bit."""
+    w = synth.WORKLOADS["window_256x256"]
+    dev = torch.device("cuda:0")
+    q, k, v = (t.to(dev) for t in synth.self_inputs(w))
+    kc, vc = (t[:, : w.n_heads].contiguous().to(dev) for t in synth.cross_inputs(synth.WORKLOADS["window_480x832"], 512))
+    out_s, out_c = torch.empty_like(q), torch.empty_like(q)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(2):  # warm-up on the capturing stream: workspace, tables, kernel attributes
+            binding.regenvc_attn_forward(q, k, v, out_s, w.T, w.H, w.W)
+            binding.regenvc_cross_attn_forward(q, kc, vc, out_c)
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        binding.regenvc_attn_forward(q, k, v, out_s, w.T, w.H, w.W)
+        binding.regenvc_cross_attn_forward(q, kc, vc, out_c)
+    # new values in the same buffers, then replay
+    w2 = synth.Workload(**{**w.__dict__, "seed": w.seed + 1000})
+    q2, k2, v2 = synth.self_inputs(w2)
+    q.copy_(q2.to(dev)); k.copy_(k2.to(dev)); v.copy_(v2.to(dev))
+    out_s.zero_(); out_c.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert binding.regenvc_device_status() == 0
+    ref_s, ref_c = torch.empty_like(q), torch.empty_like(q)
+    binding.regenvc_attn_forward(q, k, v, ref_s, w.T, w.H, w.W)
+    binding.regenvc_cross_attn_forward(q, kc, vc, ref_c)
+    torch.cuda.synchronize()
+    assert torch.equal(out_s, ref_s) and torch.equal(out_c, ref_c)
+    assert float(out_s.float().abs().max()) > 0
