@@ -118,6 +118,13 @@ __device__ __forceinline__ bool row_group_any(int g, bool flag) {
         : "memory");
     return any != 0;
 }
+// Barrier 6: the four warps of the control warpgroup.  Barrier 7, used once at start-up: the control warps arrive
+// without waiting once set-up is done, the softmax warps wait there after loading their query tiles.  (Not
+// barrier 0: the idle control warps go straight on to the __syncthreads of the tear-down, and a warp must not
+// arrive twice at a barrier whose current phase is still open.)
+__device__ __forceinline__ void control_barrier() { asm volatile("bar.sync 6, 128;" ::: "memory"); }
+__device__ __forceinline__ void setup_done_arrive() { asm volatile("bar.arrive 7, %0;" ::"n"(kThreads) : "memory"); }
+__device__ __forceinline__ void setup_done_wait() { asm volatile("bar.sync 7, %0;" ::"n"(kThreads) : "memory"); }
 // Named barrier over the kSplit warps that share the 32 rows of lane group g (barriers 2..5).
 __device__ __forceinline__ void row_group_barrier(int g) {
     asm volatile("bar.sync %0, %1;" ::"r"(2 + g), "n"(32 * kSplit) : "memory");
@@ -184,6 +191,8 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     RowExchange* xch = reinterpret_cast<RowExchange*>(base + (2 + kStages) * kTileBytes + 256);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    uint32_t tmem_base = 0;
+    const WaitCtl ctl{&bar->abort_flag, p.status, kStatusTimeout, kWaitLimitNs};
     // work item and key-tile range of this CTA
     const int n_tiles_total = p.n_kv_pad / kTile;
     int item = blockIdx.x, kv_tile0 = 0, n_tiles = n_tiles_total;
@@ -199,7 +208,11 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
     const int q0 = (item % p.pairs_per_head) * 2 * kTile;
     const bool tile1_active = q0 + kTile < p.n_q;
 
-    if (tid == 0) {
+    // Set-up is the control warpgroup's: barriers, tensor memory, descriptor prefetch.  The softmax warps do not
+    // wait for it: they fetch and rotate their query tiles first and meet the control warps at barrier 7 afterwards.
+    if (warp >= kMmaWarp) {
+      setmaxnreg_dec<kControlRegs>();
+      if (tid == kMmaWarp * 32) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_u32(&bar->kv_full[s]), 1);
             mbar_init(smem_u32(&bar->kv_empty[s]), 1);
@@ -213,25 +226,23 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         // a sticky error from an earlier kernel makes this CTA skip its work (every bounded wait falls through)
         bar->abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0) ? 1 : 0;
         fence_mbar_init();
-    }
-    if (warp == kMmaWarp) {
+      }
+      __syncwarp();
+      if (warp == kMmaWarp) {
         tmem_alloc(smem_u32(&bar->tmem_base), 512);
         tmem_relinquish();
-    }
-    if (warp == kTmaWarp && elect_one()) {
+      }
+      if (warp == kTmaWarp && elect_one()) {
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
         tma_prefetch_desc(&tmap_out);
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-
-    const uint32_t tmem_base = bar->tmem_base;
-    const WaitCtl ctl{&bar->abort_flag, p.status, kStatusTimeout, kWaitLimitNs};
-
-    if (warp >= kMmaWarp) {
-      setmaxnreg_dec<kControlRegs>();
+      }
+      __syncwarp();
+      tc_fence_before();
+      control_barrier();                 // the four control warps: set-up is complete
+      tc_fence_after();
+      setup_done_arrive();               // ... and the softmax warps may rely on it (they wait at barrier 7)
+      tmem_base = bar->tmem_base;
       if (warp == kTmaWarp) {
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
@@ -301,6 +312,9 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         if (tile1_active) load_rotate_q_tiles<kSoftmaxThreads, 2>(p, head, q0, sQ, tid);
         else load_rotate_q_tiles<kSoftmaxThreads, 1>(p, head, q0, sQ, tid);
         fence_proxy_async_smem();
+        setup_done_wait();   // barriers and tensor memory exist from here on
+        tc_fence_after();
+        tmem_base = bar->tmem_base;
         for (int t = 0; t < n_active; ++t) mbar_arrive(smem_u32(&bar->q_full[t]));
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         const float scale = p.scale_log2;
