@@ -277,3 +277,49 @@ def test_warm_calls_can_be_captured_in_a_cuda_graph_and_replayed():
     torch.cuda.synchronize()
     assert torch.equal(out_s, ref_s) and torch.equal(out_c, ref_c)
     assert float(out_s.float().abs().max()) > 0
+
+
+def test_two_host_threads_on_their_own_streams_do_not_disturb_each_other():
+    """The internal workspace is per host thread, so calls from two threads may overlap on the GPU."""
+    import threading
+
+    w = synth.WORKLOADS["window_256x256"]
+    dev = torch.device("cuda:0")
+    inputs = []
+    for i in range(2):
+        wi = synth.Workload(**{**w.__dict__, "seed": w.seed + 50 + i})
+        inputs.append([t.to(dev) for t in synth.self_inputs(wi)])
+    want = []
+    for q, k, v in inputs:
+        o = torch.empty_like(q)
+        binding.regenvc_attn_forward(q, k, v, o, w.T, w.H, w.W)
+        want.append(o)
+    torch.cuda.synchronize()
+    got = [[None] * 6 for _ in range(2)]
+    errors_seen = []
+
+    def work(i):
+        try:
+            torch.cuda.set_device(0)
+            stream = torch.cuda.Stream()
+            q, k, v = inputs[i]
+            with torch.cuda.stream(stream):
+                for r in range(6):
+                    o = torch.empty_like(q)
+                    binding.regenvc_attn_forward(q, k, v, o, w.T, w.H, w.W, stream=stream)
+                    got[i][r] = o
+            stream.synchronize()
+        except Exception as e:  # pragma: no cover
+            errors_seen.append(e)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors_seen, errors_seen
+    torch.cuda.synchronize()
+    assert binding.regenvc_device_status() == 0
+    for i in range(2):
+        for r in range(6):
+            assert torch.equal(got[i][r], want[i]), f"thread {i} call {r}"
