@@ -40,6 +40,12 @@
  *     work is enqueued, and a failing call enqueues nothing.
  *   - There is no CPU path: on a machine without an sm_100 GPU every compute
  *     entry point returns REGENVC_ERR_UNSUPPORTED or REGENVC_ERR_CUDA.
+ *   - Two environment variables, read once per process, exist for testing
+ *     and measurement: REGENVC_KERNEL=serial runs the un-pipelined bring-up
+ *     kernel instead of the pipelined one (same results within tolerance;
+ *     the block-wise calls then return REGENVC_ERR_UNSUPPORTED), and
+ *     REGENVC_SPLIT_KV=0 keeps the last wave of work items from being cut
+ *     along the keys.
  *   - Calls on one stream are ordered as usual.  Calls that overlap on the
  *     GPU (different streams) must not share a workspace: give each stream
  *     its own with regenvc_set_workspace() from the thread that launches on

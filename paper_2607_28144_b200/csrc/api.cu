@@ -226,6 +226,9 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     int rc = device_state(&dev, &st);
     if (rc != REGENVC_OK) return rc;
 
+    // the bring-up kernel (REGENVC_KERNEL=serial) only writes normalised bf16 output
+    if (serial_kernel_requested() && blk.tok_o != nullptr) return REGENVC_ERR_UNSUPPORTED;
+
     const size_t need = workspace_need(n_kv, n_heads);
     void* ws = nullptr;
     if (tl_user_ws.ptr) {

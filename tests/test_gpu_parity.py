@@ -323,3 +323,25 @@ def test_two_host_threads_on_their_own_streams_do_not_disturb_each_other():
     for i in range(2):
         for r in range(6):
             assert torch.equal(got[i][r], want[i]), f"thread {i} call {r}"
+
+
+def test_bring_up_kernel_passes_the_same_parity_cases():
+    """REGENVC_KERNEL=serial selects the un-pipelined kernel (read once per process, hence a child process): a
+    second implementation of the same operation on the GPU, checked against the oracle by the tests above, and
+    refusing the block-wise calls it does not implement."""
+    import os
+    import subprocess
+    import sys
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, REGENVC_KERNEL="serial")
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_parity.py"), "-q", "-x",
+                        "-m", "gpu", "-k", "small_shapes or test_cross_attention or brute_force or growing or "
+                        "dominating"], env=env, cwd=root, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    code = ("import torch; from paper_2607_28144_b200 import binding as b; d=torch.device('cuda:0');"
+            "q=torch.zeros((8,1,128),dtype=torch.bfloat16,device=d);"
+            "o=torch.empty((8,1,128),dtype=torch.float32,device=d); ml=torch.empty((8,1,2),dtype=torch.float32,device=d);\n"
+            "try:\n    b.regenvc_attn_partial(q,q,q,o,ml,1,2,4,0,0)\nexcept b.RegenvcError as e:\n    print('code',e.code)")
+    r = subprocess.run([sys.executable, "-c", code], env=env, cwd=root, capture_output=True, text=True, timeout=300)
+    assert f"code {binding.ERR_UNSUPPORTED}" in r.stdout, r.stdout + r.stderr
