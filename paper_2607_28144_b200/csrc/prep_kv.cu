@@ -30,6 +30,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
         // ---- K: 16 threads per row (16 B = 8 elements = 4 rotary pairs each); all loads first
         const int chunk = tid & 15;
         bool out_of_range = false;
+        __shared__ TokenPos s_pos[kTile];  // grid position of every row of the tile: one division pair per row
         uint4 raw[kTile / 16];
 #pragma unroll
         for (int it = 0; it < kTile / 16; ++it) {
@@ -38,12 +39,19 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
             if (n < p.n_kv)
                 raw[it] = __ldg(reinterpret_cast<const uint4*>(p.k + ((size_t)n * p.h + head) * kHeadDim) + chunk);
         }
+        RopeChunk rc;
+        if (p.rope) {  // uniform over the grid
+            rc = rope_chunk(p.grid, chunk);
+            if (tid < kTile) s_pos[tid] = token_pos(tile0 + tid + p.pos_offset, p.grid);
+            __syncthreads();
+        }
 #pragma unroll
         for (int it = 0; it < kTile / 16; ++it) {
-            const int n = tile0 + it * 16 + (tid >> 4);
+            const int row = it * 16 + (tid >> 4);
+            const int n = tile0 + row;
             float x[8];
             bf16x8_to_float(raw[it], x);
-            if (p.rope && n < p.n_kv) rope_rotate8(x, p.grid, token_pos(n + p.pos_offset, p.grid), chunk);
+            if (p.rope && n < p.n_kv) rope_rotate8(x, p.grid, s_pos[row], rc);
 #pragma unroll
             for (int i = 0; i < 8; ++i) out_of_range |= !(fabsf(x[i]) <= 65504.0f);
             uint4 packed;

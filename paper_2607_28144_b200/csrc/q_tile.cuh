@@ -20,6 +20,7 @@ __device__ __forceinline__ void load_rotate_q_tiles(const AttnParams& p, int hea
     constexpr int kRowsPerPass = kThreadsN / 16;
     constexpr int kPasses = kTile / kRowsPerPass;
     const int chunk = tid & 15;
+    const RopeChunk rc = rope_chunk(p.grid, chunk);
     uint4 raw[kTilesQ][kPasses];
 #pragma unroll
     for (int t = 0; t < kTilesQ; ++t)
@@ -38,7 +39,7 @@ __device__ __forceinline__ void load_rotate_q_tiles(const AttnParams& p, int hea
             const int n = q0 + t * kTile + row;
             float x[8];
             bf16x8_to_float(raw[t][it], x);
-            if (p.rope && n < p.n_q) rope_rotate8(x, p.grid, token_pos(n + p.q_pos_offset, p.grid), chunk);
+            if (p.rope && n < p.n_q) rope_rotate8(x, p.grid, token_pos(n + p.q_pos_offset, p.grid), rc);
             uint4 packed;
             packed.x = pack_f16x2(x[0], x[1]);
             packed.y = pack_f16x2(x[2], x[3]);
