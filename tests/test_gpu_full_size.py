@@ -103,3 +103,31 @@ def test_host_entry_points_at_full_size_match_the_device_path():
     binding.regenvc_cross_attn_forward_host(q, kc, vc, outc)  # pageable memory
     a, b = outc.float(), devc.float()
     _assert_close_to_device_path(a, b)
+
+
+def test_a_sustained_loop_stays_bit_exact_and_raises_no_status():
+    """Two seconds of back-to-back full-size steps (long enough for the clocks to settle under the power cap):
+    every step must reproduce the first one bit for bit, and no bounded wait may expire."""
+    import time
+
+    w = synth.WORKLOADS["window_480x832"]
+    dev = torch.device("cuda:0")
+    q, k, v = (t.to(dev) for t in synth.self_inputs(w))
+    kc, vc = (t.to(dev) for t in synth.cross_inputs(w, 512))
+    first_s, first_c = torch.empty_like(q), torch.empty_like(q)
+    binding.regenvc_attn_forward(q, k, v, first_s, w.T, w.H, w.W)
+    binding.regenvc_cross_attn_forward(q, kc, vc, first_c)
+    out_s, out_c = torch.empty_like(q), torch.empty_like(q)
+    mismatches = torch.zeros((), dtype=torch.int64, device=dev)
+    t0, steps = time.time(), 0
+    while time.time() - t0 < 2.0:
+        for _ in range(50):
+            binding.regenvc_attn_forward(q, k, v, out_s, w.T, w.H, w.W)
+            binding.regenvc_cross_attn_forward(q, kc, vc, out_c)
+            mismatches += (out_s.view(torch.int16) != first_s.view(torch.int16)).sum()
+            mismatches += (out_c.view(torch.int16) != first_c.view(torch.int16)).sum()
+            steps += 1
+        torch.cuda.synchronize()
+    assert steps >= 100
+    assert int(mismatches.item()) == 0
+    assert binding.regenvc_device_status() == 0
