@@ -237,6 +237,17 @@ int regenvc_device_status(void* stream, int* status_out);
  */
 int regenvc_debug_set_phases(int mask);
 
+/*
+ * Test aid for the bounded waits inside the kernels: enqueues one warp that
+ * waits on a barrier nothing ever completes.  After limit_us microseconds
+ * (1..100000) the wait gives up exactly as a wait in the attention kernels
+ * would, the kernel returns normally and the sticky status word holds
+ * REGENVC_ERR_TIMEOUT until regenvc_device_status() reads it.  Kernels of this
+ * library that start while the word is set skip their work (their bounded
+ * waits fall through) and leave `out` unspecified.  Nothing faults or hangs.
+ */
+int regenvc_debug_expire_wait(int limit_us, void* stream);
+
 const char* regenvc_status_string(int status);
 /* Text of the last failing CUDA call on this host thread ("" if none). */
 const char* regenvc_last_cuda_error(void);

@@ -25,7 +25,7 @@ EXPORTS = [
     "regenvc_device_status", "regenvc_status_string", "regenvc_last_cuda_error", "regenvc_version",
     "regenvc_kernel_launch_count", "regenvc_shutdown", "regenvc_debug_set_phases",
     "regenvc_cross_attn_forward_static", "regenvc_attn_partial", "regenvc_attn_merge",
-    "regenvc_ulysses_scatter_heads", "regenvc_ulysses_gather_heads",
+    "regenvc_ulysses_scatter_heads", "regenvc_ulysses_gather_heads", "regenvc_debug_expire_wait",
 ]
 
 _lib = None
@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
     L.regenvc_version.restype = ctypes.c_char_p
     L.regenvc_kernel_launch_count.argtypes = []
     L.regenvc_kernel_launch_count.restype = ctypes.c_ulonglong
+    L.regenvc_debug_expire_wait.argtypes = [i32, vp]
+    L.regenvc_debug_expire_wait.restype = i32
     L.regenvc_debug_set_phases.argtypes = [i32]
     L.regenvc_debug_set_phases.restype = i32
     L.regenvc_shutdown.argtypes = []
@@ -276,6 +278,11 @@ def regenvc_kernel_launch_count() -> int:
 def regenvc_debug_set_phases(mask: int):
     """Profiling aid: 1 = preparation pass only, 2 = attention kernel only, 3 = both (default)."""
     _check(lib().regenvc_debug_set_phases(mask))
+
+
+def regenvc_debug_expire_wait(limit_us: int = 500, stream=None):
+    """Test aid: one warp waits limit_us on a barrier nothing completes; the sticky status becomes ERR_TIMEOUT."""
+    _check(lib().regenvc_debug_expire_wait(int(limit_us), _stream(stream)))
 
 
 def regenvc_shutdown():

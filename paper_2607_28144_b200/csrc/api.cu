@@ -661,6 +661,22 @@ int regenvc_debug_set_phases(int mask) {
     return REGENVC_OK;
 }
 
+int regenvc_debug_expire_wait(int limit_us, void* stream) {
+    if (limit_us < 1 || limit_us > 100000) return REGENVC_ERR_BAD_SHAPE;
+    int* status = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        int dev = 0;
+        DeviceState* st = nullptr;
+        int rc = device_state(&dev, &st);
+        if (rc != REGENVC_OK) return rc;
+        status = st->status;
+    }
+    CUDA_TRY(launch_expire_wait(status, (unsigned long long)limit_us * 1000ull, (cudaStream_t)stream));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return REGENVC_OK;
+}
+
 const char* regenvc_status_string(int status) {
     switch (status) {
         case REGENVC_OK: return "ok";

@@ -101,6 +101,9 @@ struct ReshardParams {
 cudaError_t launch_scatter_heads(const ReshardParams& p, int sm_count, cudaStream_t stream);
 cudaError_t launch_gather_heads(const ReshardParams& p, int sm_count, cudaStream_t stream);
 
+// One warp that waits `limit_ns` on a barrier nothing completes and then records kStatusTimeout (test aid).
+cudaError_t launch_expire_wait(int* status, unsigned long long limit_ns, cudaStream_t stream);
+
 // Launchers (each returns the launch error, enqueues on `stream`).
 cudaError_t launch_prep_kv(const PrepParams& p, cudaStream_t stream);
 cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
