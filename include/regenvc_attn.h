@@ -4,9 +4,9 @@
  * The operation is the attention step of the paper's real-time decoder: every
  * block of the four-step diffusion transformer runs exact, non-causal
  * multi-head softmax attention over the whole flattened T x H x W latent-token
- * sequence of a 25-frame window (Sec. 3.5: after the Ulysses exchange each
- * device "computes exact attention over the full sequence for a subset of
- * heads"; here that is done for all heads on one GPU with no sharding), and
+ * sequence of a 25-frame window (Sec. 3.5: after the Ulysses exchange a
+ * device holds some of the heads and attends over the whole sequence for
+ * them; here that is done for all heads on one GPU with no sharding), and
  * cross-attention of the same queries to the short, precomputed text/image
  * conditioning key/value tensors (Sec. 3.9).  The backbone's 3D rotary
  * position embedding is applied to queries and keys inside the call.
@@ -98,8 +98,8 @@ int regenvc_cross_attn_forward(const void* q, const void* k, const void* v, void
 
 /*
  * Block-wise attention for sequence-parallel use (Sec. 3.5: Ring attention streams key/value blocks around
- * the devices and combines the per-block results "in an online-softmax fashion"; the result equals
- * unsharded attention up to reduction order).
+ * the devices and combines the per-block results by the online-softmax rule; the result is unsharded
+ * attention, only summed in another order).
  *
  * regenvc_attn_partial(): attention of a contiguous range of query tokens against ONE contiguous range of
  * key/value tokens of the same T x H x W grid, left unnormalised.

@@ -4,8 +4,8 @@
  * A plain, slow, fp64 CPU statement of what the decoder's attention step
  * computes: exact (non-causal, unmasked) multi-head softmax attention of every
  * latent token against the whole token sequence of one window (the paper's
- * Sec. 3.5: each device "computes exact attention over the full sequence for
- * a subset of heads"), with the backbone's 3D rotary position embedding on the
+ * Sec. 3.5: once the heads have been redistributed, a device attends over the
+ * whole sequence for its heads), with the backbone's 3D rotary position embedding on the
  * queries and keys, plus the cross-attention of the same queries against the
  * short, precomputed conditioning key/value tensors of Sec. 3.9.
  *

@@ -1,6 +1,6 @@
 """Block-wise attention: partial results over key/value blocks, merged by the online-softmax rule, reproduce
-unsharded attention (the paper's Sec. 3.5: sequence parallelism "preserves exact attention ... up to reduction
-order").  Checked against the fp64 oracle of the WHOLE sequence, so a wrong rotary offset of a block, a wrong
+unsharded attention (the paper's Sec. 3.5: its sequence parallelism changes only the order of the sums, not the
+result).  Checked against the fp64 oracle of the WHOLE sequence, so a wrong rotary offset of a block, a wrong
 reference or a wrong merge weight all show."""
 import numpy as np
 import pytest

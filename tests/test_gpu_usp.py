@@ -1,6 +1,6 @@
 """Ulysses x Ring on one GPU: the resharding kernels against their index definition (bit-exact), and the whole
 scheme, all ranks executed one after another, against the fp64 oracle of the UNSHARDED sequence (Sec. 3.5: the
-parallel form is exact attention up to reduction order)."""
+parallel form changes the order of the sums, nothing else)."""
 import numpy as np
 import pytest
 import torch
