@@ -153,7 +153,7 @@ int regenvc_ulysses_gather_heads(const void* x_heads, void* const* dst, const in
  * staged by the driver).  The call copies q, k, v to device staging buffers
  * that the library owns and reuses, runs the device path, copies the result
  * back into `out` and waits for `stream` before returning.  K and V are
- * copied first; the query rows follow in up to 8 blocks of at least one wave
+ * copied first; the query rows follow in up to 8 blocks of about one wave
  * of work items, and the library's own copy-in and copy-out streams overlap
  * the transfer of a block with the attention of the previous one (all of it
  * ordered after the work already on `stream`).  The result equals the device
