@@ -40,12 +40,6 @@
  *     work is enqueued, and a failing call enqueues nothing.
  *   - There is no CPU path: on a machine without an sm_100 GPU every compute
  *     entry point returns REGENVC_ERR_UNSUPPORTED or REGENVC_ERR_CUDA.
- *   - Two environment variables, read once per process, exist for testing
- *     and measurement: REGENVC_KERNEL=serial runs the un-pipelined bring-up
- *     kernel instead of the pipelined one (same results within tolerance;
- *     the block-wise calls then return REGENVC_ERR_UNSUPPORTED), and
- *     REGENVC_SPLIT_KV=0 keeps the last wave of work items from being cut
- *     along the keys.
  *   - Calls on one stream are ordered as usual.  Calls that overlap on the
  *     GPU (different streams) must not share a workspace: give each stream
  *     its own with regenvc_set_workspace() from the thread that launches on
@@ -193,10 +187,18 @@ int regenvc_cross_attn_forward_host(const void* q, const void* k, const void* v,
  *     events.  regenvc_set_workspace() has no effect here.
  *   - Device-side conditions of these calls (an input beyond the fp16 range, an expired bounded wait) are
  *     recorded in a status word that is also part of the image, not in the one regenvc_device_status() reads.
+ *     The word is sticky: while it is set, later calls of this entry point on the device skip their work and
+ *     leave `out` unspecified although they return REGENVC_OK.  regenvc_static_device_status() waits for
+ *     `stream`, reports the word in *status_out (REGENVC_OK, REGENVC_ERR_RANGE or REGENVC_ERR_TIMEOUT) and
+ *     clears it; it allocates nothing either (a stream synchronisation and a 4-byte copy).  A real-time loop
+ *     should read it once per window, after the window's last call.
+ *   - The call enqueues two kernels.  Arguments are validated before the first; if the launch of the second
+ *     fails (REGENVC_ERR_CUDA), the first, which only rewrites the scratch array, has already been enqueued.
  */
 #define REGENVC_STATIC_SCRATCH_BYTES (16u << 20)
 int regenvc_cross_attn_forward_static(const void* q, const void* k, const void* v, void* out,
                                       int n_q, int n_kv, int n_heads, int head_dim, void* stream);
+int regenvc_static_device_status(void* stream, int* status_out);
 
 /*
  * Scratch memory.  Each call first rewrites the keys and values into

@@ -24,7 +24,7 @@ EXPORTS = [
     "regenvc_cross_attn_forward_host", "regenvc_workspace_bytes", "regenvc_set_workspace",
     "regenvc_device_status", "regenvc_status_string", "regenvc_last_cuda_error", "regenvc_version",
     "regenvc_kernel_launch_count", "regenvc_shutdown", "regenvc_debug_set_phases",
-    "regenvc_cross_attn_forward_static", "regenvc_attn_partial", "regenvc_attn_merge",
+    "regenvc_cross_attn_forward_static", "regenvc_static_device_status", "regenvc_attn_partial", "regenvc_attn_merge",
     "regenvc_ulysses_scatter_heads", "regenvc_ulysses_gather_heads", "regenvc_debug_expire_wait",
 ]
 
@@ -72,6 +72,8 @@ def lib() -> ctypes.CDLL:
     L.regenvc_set_workspace.restype = i32
     L.regenvc_device_status.argtypes = [vp, ctypes.POINTER(i32)]
     L.regenvc_device_status.restype = i32
+    L.regenvc_static_device_status.argtypes = [vp, ctypes.POINTER(i32)]
+    L.regenvc_static_device_status.restype = i32
     L.regenvc_status_string.argtypes = [i32]
     L.regenvc_status_string.restype = ctypes.c_char_p
     L.regenvc_last_cuda_error.argtypes = []
@@ -264,6 +266,13 @@ def regenvc_device_status(stream=None) -> int:
     """Waits for ``stream`` and returns (then clears) the sticky device status."""
     st = ctypes.c_int(0)
     _check(lib().regenvc_device_status(_stream(stream), ctypes.byref(st)))
+    return st.value
+
+
+def regenvc_static_device_status(stream=None) -> int:
+    """Waits for ``stream`` and returns (then clears) the status word of the allocation-free entry point."""
+    st = ctypes.c_int(0)
+    _check(lib().regenvc_static_device_status(_stream(stream), ctypes.byref(st)))
     return st.value
 
 

@@ -13,11 +13,6 @@
 #include "../../include/regenvc_attn.h"
 #include "common.cuh"
 
-namespace regenvc {
-cudaError_t configure_attn_serial();
-cudaError_t launch_attn_serial(const CUtensorMap&, const CUtensorMap&, const AttnParams&, cudaStream_t);
-cudaError_t configure_attn_pipelined();
-}  // namespace regenvc
 
 namespace {
 
@@ -26,6 +21,14 @@ using namespace regenvc;
 struct Buf {
     void* ptr = nullptr;
     size_t bytes = 0;
+};
+// A default workspace remembers the stream of its last user and an event recorded behind that user's kernels,
+// so that a call on another stream is ordered after them instead of overwriting operands still being read.
+struct Workspace {
+    Buf buf;
+    cudaEvent_t last_use = nullptr;
+    cudaStream_t last_stream = nullptr;
+    bool used = false;
 };
 struct RopeEntry {
     int T, H, W;
@@ -46,7 +49,7 @@ struct DeviceState {
     int* status = nullptr;
     int sm_count = 0;
     std::vector<RopeEntry> ropes;
-    std::map<std::thread::id, Buf> workspace;
+    std::map<std::thread::id, Workspace> workspace;
     std::map<std::thread::id, std::vector<Buf>> staging;  // q, k, v, out
     std::map<std::thread::id, HostPipe> pipes;
 };
@@ -68,27 +71,12 @@ int cuda_fail(cudaError_t e, const char* what) {
     (void)cudaGetLastError();
     return REGENVC_ERR_CUDA;
 }
+void launched() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 #define CUDA_TRY(expr)                                   \
     do {                                                 \
         cudaError_t e_ = (expr);                         \
         if (e_ != cudaSuccess) return cuda_fail(e_, #expr); \
     } while (0)
-
-bool serial_kernel_requested() {
-    static const bool serial = [] {
-        const char* e = std::getenv("REGENVC_KERNEL");
-        return e && std::strcmp(e, "serial") == 0;
-    }();
-    return serial;
-}
-
-bool split_disabled() {
-    static const bool off = [] {
-        const char* e = std::getenv("REGENVC_SPLIT_KV");
-        return e && std::strcmp(e, "0") == 0;
-    }();
-    return off;
-}
 
 bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
     const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
@@ -134,7 +122,6 @@ int device_state(int* dev_out, DeviceState** st_out) {
                 }
                 g_encode = (EncodeTiledFn)fn;
             }
-            CUDA_TRY(configure_attn_serial());
             CUDA_TRY(configure_attn_pipelined());
             CUDA_TRY(cudaMalloc(&st.status, sizeof(int)));
             CUDA_TRY(cudaMemset(st.status, 0, sizeof(int)));
@@ -144,6 +131,33 @@ int device_state(int* dev_out, DeviceState** st_out) {
     *dev_out = dev;
     *st_out = &st;
     return st.supported ? REGENVC_OK : REGENVC_ERR_UNSUPPORTED;
+}
+
+// True when `stream` is being captured into a graph (or its state cannot be queried): events of the library
+// are then left alone, and ordering against other streams stays with the caller.
+bool capturing(cudaStream_t stream) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return true;
+    }
+    return cs != cudaStreamCaptureStatusNone;
+}
+
+// Two calls of one host thread on different streams would share the thread's default workspace while both are
+// in flight.  The second one is made to wait (on the GPU, not on the host) for the first one's kernels.
+int order_after_last_user(Workspace& w, cudaStream_t stream) {
+    if (!w.used || w.last_stream == stream || capturing(stream)) return REGENVC_OK;
+    CUDA_TRY(cudaStreamWaitEvent(stream, w.last_use, 0));
+    return REGENVC_OK;
+}
+int note_use(Workspace& w, cudaStream_t stream) {
+    if (capturing(stream)) return REGENVC_OK;
+    if (!w.last_use) CUDA_TRY(cudaEventCreateWithFlags(&w.last_use, cudaEventDisableTiming));
+    CUDA_TRY(cudaEventRecord(w.last_use, stream));
+    w.last_stream = stream;
+    w.used = true;
+    return REGENVC_OK;
 }
 
 int grow(Buf& b, size_t bytes) {
@@ -226,19 +240,19 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     int rc = device_state(&dev, &st);
     if (rc != REGENVC_OK) return rc;
 
-    // the bring-up kernel (REGENVC_KERNEL=serial) only writes normalised bf16 output
-    if (serial_kernel_requested() && blk.tok_o != nullptr) return REGENVC_ERR_UNSUPPORTED;
-
     const size_t need = workspace_need(n_kv, n_heads);
     void* ws = nullptr;
+    Workspace* own = nullptr;  // the library's workspace of this thread, when the caller supplied none
     if (tl_user_ws.ptr) {
         if (tl_user_ws.bytes < need) return REGENVC_ERR_WORKSPACE;
         ws = tl_user_ws.ptr;
     } else {
-        Buf& b = st->workspace[std::this_thread::get_id()];
-        rc = grow(b, need);
+        own = &st->workspace[std::this_thread::get_id()];
+        rc = grow(own->buf, need);
         if (rc != REGENVC_OK) return rc;
-        ws = b.ptr;
+        ws = own->buf.ptr;
+        rc = order_after_last_user(*own, stream);
+        if (rc != REGENVC_OK) return rc;
     }
     const int kv_pad = round_up(n_kv, kTile);
     __half* kp = reinterpret_cast<__half*>(ws);
@@ -271,9 +285,9 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     const int phases = blk.phases >= 0 ? blk.phases : tl_phases;
     if (phases & 1) {
         CUDA_TRY(launch_prep_kv(pp, stream));
-        g_launches.fetch_add(1, std::memory_order_relaxed);
+        launched();
     }
-    if (!(phases & 2)) return REGENVC_OK;
+    if (!(phases & 2)) return own ? note_use(*own, stream) : REGENVC_OK;
 
     AttnParams ap;
     ap.q = reinterpret_cast<const __nv_bfloat16*>(q);
@@ -301,7 +315,7 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     ap.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + operand_bytes(n_kv, n_heads));
     ap.part_ml = reinterpret_cast<float2*>(ap.part_o + (size_t)kMaxPieceCtas * 2 * kTile * kHeadDim);
     const int rem = n_items % st->sm_count;
-    if (rem > 0 && st->sm_count <= kMaxPieceCtas && !split_disabled() && blk.tok_o == nullptr) {
+    if (rem > 0 && st->sm_count <= kMaxPieceCtas && blk.tok_o == nullptr) {
         int k = st->sm_count / rem;
         if (k > 8) k = 8;
         if (k > n_tiles / 4) k = n_tiles / 4;
@@ -311,18 +325,13 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
             ap.n_full_items = n_items - rem;
         }
     }
-    if (serial_kernel_requested()) {
-        CUDA_TRY(launch_attn_serial(tmap_k, tmap_v, ap, stream));
-        g_launches.fetch_add(1, std::memory_order_relaxed);
-        return REGENVC_OK;
-    }
     // out seen as [n_q rows][n_heads * 128 columns] bf16 for the tiled stores of finished query tiles
     CUtensorMap tmap_out;
     rc = make_tmap(&tmap_out, out != nullptr ? out : const_cast<void*>(q), (uint64_t)n_heads * kHeadDim, (uint64_t)n_q,
                    (uint64_t)n_heads * kHeadDim * sizeof(__nv_bfloat16), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     if (rc != REGENVC_OK) return rc;
     CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, ap, stream));
-    g_launches.fetch_add(1, std::memory_order_relaxed);
+    launched();
     if (ap.split_k > 1) {
         MergeParams mp;
         mp.part_o = ap.part_o;
@@ -335,9 +344,9 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
         mp.split_k = ap.split_k;
         mp.n_split_items = n_items - ap.n_full_items;
         CUDA_TRY(launch_merge_partials(mp, stream));
-        g_launches.fetch_add(1, std::memory_order_relaxed);
+        launched();
     }
-    return REGENVC_OK;
+    return own ? note_use(*own, stream) : REGENVC_OK;
 }
 
 int make_pipe(HostPipe& hp) {
@@ -439,6 +448,11 @@ int check_self_args(int T, int H, int W, float theta, long long* n_out) {
 
 }  // namespace
 
+namespace regenvc {
+void count_launch() { launched(); }
+int record_cuda_failure(cudaError_t e, const char* what) { return cuda_fail(e, what); }
+}  // namespace regenvc
+
 extern "C" {
 
 int regenvc_attn_forward(const void* q, const void* k, const void* v, void* out, int T, int H, int W, int n_heads,
@@ -511,6 +525,7 @@ int regenvc_attn_merge(const void* const* o_parts, const void* const* mls, int n
                        int n_heads, int head_dim, void* stream) {
     if (!o_parts || !mls || !out) return REGENVC_ERR_NULL_POINTER;
     if (n_parts < 1 || n_parts > kMaxMergeParts || n_q < 1 || n_heads < 1) return REGENVC_ERR_BAD_SHAPE;
+    if (n_q > (1 << 30) || n_heads > 65535 || (long long)n_q * n_heads >= (1ll << 31)) return REGENVC_ERR_BAD_SHAPE;
     if (head_dim != kHeadDim) return REGENVC_ERR_UNSUPPORTED;
     TokenMergeParams mp;
     const size_t rows = (size_t)n_q * n_heads;
@@ -535,7 +550,7 @@ int regenvc_attn_merge(const void* const* o_parts, const void* const* mls, int n
         if (rc != REGENVC_OK) return rc;
     }
     CUDA_TRY(launch_merge_token_partials(mp, (cudaStream_t)stream));
-    g_launches.fetch_add(1, std::memory_order_relaxed);
+    launched();
     return REGENVC_OK;
 }
 
@@ -575,7 +590,7 @@ int regenvc_ulysses_scatter_heads(const void* x_local, void* const* dst, int wor
     }
     if (n_local == 0) return REGENVC_OK;
     CUDA_TRY(launch_scatter_heads(rp, sm_count, (cudaStream_t)stream));
-    g_launches.fetch_add(1, std::memory_order_relaxed);
+    launched();
     return REGENVC_OK;
 }
 
@@ -621,7 +636,7 @@ int regenvc_ulysses_gather_heads(const void* x_heads, void* const* dst, const in
     }
     if (total == 0) return REGENVC_OK;
     CUDA_TRY(launch_gather_heads(rp, sm_count, (cudaStream_t)stream));
-    g_launches.fetch_add(1, std::memory_order_relaxed);
+    launched();
     return REGENVC_OK;
 }
 
@@ -674,7 +689,7 @@ int regenvc_debug_expire_wait(int limit_us, void* stream) {
         status = st->status;
     }
     CUDA_TRY(launch_expire_wait(status, (unsigned long long)limit_us * 1000ull, (cudaStream_t)stream));
-    g_launches.fetch_add(1, std::memory_order_relaxed);
+    launched();
     return REGENVC_OK;
 }
 
@@ -714,7 +729,10 @@ void regenvc_shutdown(void) {
         DeviceState& st = kv.second;
         if (st.status) cudaFree(st.status);
         for (RopeEntry& e : st.ropes) cudaFree(e.dev);
-        for (auto& w : st.workspace) cudaFree(w.second.ptr);
+        for (auto& w : st.workspace) {
+            cudaFree(w.second.buf.ptr);
+            if (w.second.last_use) cudaEventDestroy(w.second.last_use);
+        }
         for (auto& s : st.staging)
             for (Buf& b : s.second) cudaFree(b.ptr);
         for (auto& hp : st.pipes) {

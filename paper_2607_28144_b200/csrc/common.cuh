@@ -104,6 +104,12 @@ cudaError_t launch_gather_heads(const ReshardParams& p, int sm_count, cudaStream
 // One warp that waits `limit_ns` on a barrier nothing completes and then records kStatusTimeout (test aid).
 cudaError_t launch_expire_wait(int* status, unsigned long long limit_ns, cudaStream_t stream);
 
+// Host-side bookkeeping shared by the files that implement entry points: every kernel launch is counted
+// (regenvc_kernel_launch_count), and a failing CUDA call leaves its text for regenvc_last_cuda_error(), clears the
+// runtime's error state and maps to REGENVC_ERR_CUDA.
+void count_launch();
+int record_cuda_failure(cudaError_t e, const char* what);
+
 // Launchers (each returns the launch error, enqueues on `stream`).
 cudaError_t launch_prep_kv(const PrepParams& p, cudaStream_t stream);
 cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,

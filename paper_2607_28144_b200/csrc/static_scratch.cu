@@ -35,27 +35,34 @@ EncodeTiledFn g_static_encode = nullptr;
 // allocates device memory.
 int static_setup(StaticDevice** out) {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return REGENVC_ERR_CUDA;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_failure(e, "cudaGetDevice");
     auto it = g_static_dev.find(dev);
     if (it != g_static_dev.end()) {
         *out = &it->second;
         return REGENVC_OK;
     }
     int major = 0;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return REGENVC_ERR_CUDA;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return record_cuda_failure(e, "cudaDeviceGetAttribute");
     if (major != 10) return REGENVC_ERR_UNSUPPORTED;
     if (!g_static_encode) {
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
-            qres != cudaDriverEntryPointSuccess)
-            return REGENVC_ERR_CUDA;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess)
+            return record_cuda_failure(e == cudaSuccess ? cudaErrorNotSupported : e, "cuTensorMapEncodeTiled lookup");
         g_static_encode = (EncodeTiledFn)fn;
     }
-    if (configure_attn_pipelined() != cudaSuccess) return REGENVC_ERR_CUDA;
+    e = configure_attn_pipelined();
+    if (e != cudaSuccess) return record_cuda_failure(e, "kernel attributes of the attention kernel");
     StaticDevice d;
-    if (cudaGetSymbolAddress((void**)&d.scratch, g_static_scratch) != cudaSuccess || !d.scratch) return REGENVC_ERR_CUDA;
-    if (cudaGetSymbolAddress((void**)&d.status, g_static_status) != cudaSuccess || !d.status) return REGENVC_ERR_CUDA;
+    e = cudaGetSymbolAddress((void**)&d.scratch, g_static_scratch);
+    if (e != cudaSuccess || !d.scratch)
+        return record_cuda_failure(e == cudaSuccess ? cudaErrorInvalidSymbol : e, "cudaGetSymbolAddress(scratch array)");
+    e = cudaGetSymbolAddress((void**)&d.status, g_static_status);
+    if (e != cudaSuccess || !d.status)
+        return record_cuda_failure(e == cudaSuccess ? cudaErrorInvalidSymbol : e, "cudaGetSymbolAddress(status word)");
     *out = &(g_static_dev[dev] = d);
     return REGENVC_OK;
 }
@@ -70,11 +77,11 @@ int encode_map(CUtensorMap* m, CUtensorMapDataType type, void* base, uint64_t in
     const cuuint64_t gstride[1] = {row_bytes};
     const cuuint32_t box[2] = {64, 128};
     const cuuint32_t estr[2] = {1, 1};
-    return g_static_encode(m, type, 2, base, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS
-               ? REGENVC_OK
-               : REGENVC_ERR_CUDA;
+    if (g_static_encode(m, type, 2, base, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return record_cuda_failure(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return REGENVC_OK;
 }
 
 }  // namespace
@@ -124,7 +131,9 @@ extern "C" int regenvc_cross_attn_forward_static(const void* q, const void* k, c
     pp.grid = RopeGrid{nullptr, 1, 1, 1};
     pp.pos_offset = 0;
     pp.status = dev->status;
-    if (launch_prep_kv(pp, (cudaStream_t)stream) != cudaSuccess) return REGENVC_ERR_CUDA;
+    cudaError_t e = launch_prep_kv(pp, (cudaStream_t)stream);
+    if (e != cudaSuccess) return record_cuda_failure(e, "launch of the key/value preparation kernel");
+    count_launch();
 
     AttnParams ap;
     ap.q = reinterpret_cast<const __nv_bfloat16*>(q);
@@ -147,6 +156,27 @@ extern "C" int regenvc_cross_attn_forward_static(const void* q, const void* k, c
     ap.tok_ml = nullptr;
     ap.part_o = nullptr;
     ap.part_ml = nullptr;
-    if (launch_attn_pipelined(tmap_k, tmap_v, tmap_out, ap, (cudaStream_t)stream) != cudaSuccess) return REGENVC_ERR_CUDA;
+    e = launch_attn_pipelined(tmap_k, tmap_v, tmap_out, ap, (cudaStream_t)stream);
+    if (e != cudaSuccess) return record_cuda_failure(e, "launch of the attention kernel");
+    count_launch();
+    return REGENVC_OK;
+}
+
+extern "C" int regenvc_static_device_status(void* stream, int* status_out) {
+    if (!status_out) return REGENVC_ERR_NULL_POINTER;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    StaticDevice* dev = nullptr;
+    int rc = static_setup(&dev);
+    if (rc != REGENVC_OK) return rc;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return record_cuda_failure(e, "cudaStreamSynchronize");
+    int h = 0;
+    e = cudaMemcpy(&h, dev->status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return record_cuda_failure(e, "cudaMemcpy(status word of the built-in scratch)");
+    if (h != 0) {
+        e = cudaMemset(dev->status, 0, sizeof(int));
+        if (e != cudaSuccess) return record_cuda_failure(e, "cudaMemset(status word of the built-in scratch)");
+    }
+    *status_out = h;
     return REGENVC_OK;
 }

@@ -75,6 +75,16 @@ def test_argument_validation_happens_before_any_cuda_call(L):
         assert host(None, k, v, o, 1, 1, 1, 1, 128, 1e4, None) == binding.ERR_NULL_POINTER
         assert host(q, k, v, o, 1, 1, 1, 1, 32, 1e4, None) == binding.ERR_UNSUPPORTED
     assert L.regenvc_cross_attn_forward_host(q, k, v, q, 4, 4, 1, 128, None) == binding.ERR_ALIASING
+    # the merge of partial results applies the same size limits as the calls that produce them
+    ptrs = (ctypes.c_void_p * 2)(0x50000, 0x60000)
+    m = L.regenvc_attn_merge
+    assert m(ptrs, ptrs, 2, o, (1 << 30) + 1, 1, 128, None) == binding.ERR_BAD_SHAPE
+    assert m(ptrs, ptrs, 2, o, 1 << 20, 1 << 11, 128, None) == binding.ERR_BAD_SHAPE   # n_q * n_heads = 2^31
+    assert m(ptrs, ptrs, 2, o, 4, 70000, 128, None) == binding.ERR_BAD_SHAPE
+    assert m(ptrs, ptrs, 9, o, 4, 1, 128, None) == binding.ERR_BAD_SHAPE
+    assert m(ptrs, ptrs, 2, o, 4, 1, 64, None) == binding.ERR_UNSUPPORTED
+    assert m(ptrs, ptrs, 2, None, 4, 1, 128, None) == binding.ERR_NULL_POINTER
+    assert L.regenvc_static_device_status(None, None) == binding.ERR_NULL_POINTER
     assert L.regenvc_set_workspace(0x1001, 1 << 20) == binding.ERR_WORKSPACE
     assert L.regenvc_set_workspace(None, 0) == binding.OK
     assert L.regenvc_device_status(None, None) == binding.ERR_NULL_POINTER

@@ -103,6 +103,17 @@ def test_host_entry_points_at_full_size_match_the_device_path():
     binding.regenvc_cross_attn_forward_host(q, kc, vc, outc)  # pageable memory
     a, b = outc.float(), devc.float()
     _assert_close_to_device_path(a, b)
+    # ... and, since this is the path the end-to-end timing runs, against the oracle itself on the sampled rows
+    # (which include both sides of the host path's block boundaries: the samples straddle every multiple of 256
+    # near the middle of the sequence and the whole ragged tail)
+    rows = synth.sample_rows(w.n_tokens, w.H, w.W, seed=w.seed)
+    qb, kb, vb = synth.bits(q), synth.bits(k), synth.bits(v)
+    max_v, max_vc = float(v.float().abs().max()), float(vc.float().abs().max())
+    for head in (0, 5, w.n_heads - 1):
+        ref = oracle.self_attn_head(qb, kb, vb, w.T, w.H, w.W, head, w.theta, rows=rows)
+        assert_parity(out[rows, head].double().numpy(), ref, max_v, f"host self-attention head {head}")
+        ref = oracle.cross_attn_head(qb, synth.bits(kc), synth.bits(vc), head, rows=rows)
+        assert_parity(outc[rows, head].double().numpy(), ref, max_vc, f"host cross-attention head {head}")
 
 
 def test_a_sustained_loop_stays_bit_exact_and_raises_no_status():

@@ -194,6 +194,26 @@ def test_scores_that_grow_along_the_sequence_force_reference_updates(growth):
     assert_parity(gpu, ref, float(v.float().abs().max()), f"growing scores x{growth}")
 
 
+@pytest.mark.parametrize("amp", [3.5, 4.0, 5.0])
+@pytest.mark.parametrize("key", [128 + 4, 128 + 13, 256 + 37, 128 + 0, 256 + 28])
+def test_one_key_far_above_the_reference_of_the_earlier_tiles(key, amp):
+    """Flat scores in the first key tile, then ONE key whose score lies 200 to 400 log2 units above them, placed
+    both in columns whose exponential is evaluated by the polynomial (key index mod 16 in {4, 5, 12, 13}) and in
+    MUFU columns: the jump must raise the reference (not wrap the polynomial's exponent field), so every output
+    row equals that key's value vector."""
+    n_q, n_kv, h = 200, 300, 2
+    rng = np.random.default_rng(41)
+    q = synth.from_f32(np.full((n_q, h, D), amp, dtype=np.float32))
+    k = np.zeros((n_kv, h, D), dtype=np.float32)
+    k[key] = amp                       # score 128 amp^2, times log2(e)/sqrt(128): 200 / 261 / 408 log2 units
+    k = synth.from_f32(k)
+    v = _rand(rng, n_kv, h)
+    gpu = f64(run_gpu_cross(q, k, v))
+    ref = oracle.cross_attention(synth.bits(q), synth.bits(k), synth.bits(v))
+    np.testing.assert_allclose(ref, np.broadcast_to(f64(v)[key], ref.shape), atol=1e-12)
+    assert_parity(gpu, ref, float(v.float().abs().max()), f"jump at key {key}, amplitude {amp}")
+
+
 def test_heads_are_independent_on_the_gpu():
     T, H, W, h = 2, 9, 10, 4
     N = T * H * W
@@ -325,23 +345,25 @@ def test_two_host_threads_on_their_own_streams_do_not_disturb_each_other():
             assert torch.equal(got[i][r], want[i]), f"thread {i} call {r}"
 
 
-def test_bring_up_kernel_passes_the_same_parity_cases():
-    """REGENVC_KERNEL=serial selects the un-pipelined kernel (read once per process, hence a child process): a
-    second implementation of the same operation on the GPU, checked against the oracle by the tests above, and
-    refusing the block-wise calls it does not implement."""
-    import os
-    import subprocess
-    import sys
-
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    env = dict(os.environ, REGENVC_KERNEL="serial")
-    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_parity.py"), "-q", "-x",
-                        "-m", "gpu", "-k", "small_shapes or test_cross_attention or brute_force or growing or "
-                        "dominating"], env=env, cwd=root, capture_output=True, text=True, timeout=900)
-    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
-    code = ("import torch; from paper_2607_28144_b200 import binding as b; d=torch.device('cuda:0');"
-            "q=torch.zeros((8,1,128),dtype=torch.bfloat16,device=d);"
-            "o=torch.empty((8,1,128),dtype=torch.float32,device=d); ml=torch.empty((8,1,2),dtype=torch.float32,device=d);\n"
-            "try:\n    b.regenvc_attn_partial(q,q,q,o,ml,1,2,4,0,0)\nexcept b.RegenvcError as e:\n    print('code',e.code)")
-    r = subprocess.run([sys.executable, "-c", code], env=env, cwd=root, capture_output=True, text=True, timeout=300)
-    assert f"code {binding.ERR_UNSUPPORTED}" in r.stdout, r.stdout + r.stderr
+def test_one_thread_two_streams_share_the_default_workspace_safely():
+    """A self-attention call on one stream and a cross-attention call on another, both from this thread, use the
+    same default workspace: the library orders the second behind the first on the GPU, so both results equal
+    those of the same calls made one after the other."""
+    w = synth.WORKLOADS["window_256x256"]
+    dev = torch.device("cuda:0")
+    q, k, v = (t.to(dev) for t in synth.self_inputs(w))
+    kc, vc = (t[:, : w.n_heads].contiguous().to(dev) for t in synth.cross_inputs(synth.WORKLOADS["window_480x832"], 512))
+    want_s, want_c = torch.empty_like(q), torch.empty_like(q)
+    binding.regenvc_attn_forward(q, k, v, want_s, w.T, w.H, w.W)
+    binding.regenvc_cross_attn_forward(q, kc, vc, want_c)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Stream(), torch.cuda.Stream()
+    for _ in range(20):
+        got_s, got_c = torch.full_like(q, float("nan")), torch.full_like(q, float("nan"))
+        torch.cuda.synchronize()
+        binding.regenvc_attn_forward(q, k, v, got_s, w.T, w.H, w.W, stream=a)
+        binding.regenvc_cross_attn_forward(q, kc, vc, got_c, stream=b)
+        binding.regenvc_attn_forward(q, k, v, got_s, w.T, w.H, w.W, stream=a)
+        torch.cuda.synchronize()
+        assert torch.equal(got_s, want_s) and torch.equal(got_c, want_c)
+    assert binding.regenvc_device_status() == 0

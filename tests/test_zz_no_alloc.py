@@ -6,7 +6,9 @@ synchronise the device and stall the other streams, or a process whose framework
 memory.  For them regenvc_cross_attn_forward_static() keeps its operand scratch in a fixed array inside the
 library.  This test calls it through the C ABI twice in a row (the second time with a shorter key sequence,
 so that stale operands of the first call are still in the array) and checks each result against the
-ordinary entry point, within the tolerance the parity tests use.
+ordinary entry point and against the fp64 oracle, within the tolerance the parity tests use.  A second test
+covers the entry point's own sticky status word: an out-of-range input is reported, the report clears the
+word, and the next call computes normally again.
 """
 import ctypes
 
@@ -14,8 +16,9 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2607_28144_b200 import binding, synth
-from parity_util import MAX_ERR_FACTOR, MRE_LIMIT
+from parity_util import MAX_ERR_FACTOR, MRE_LIMIT, assert_parity
 
 pytestmark = pytest.mark.gpu
 
@@ -55,6 +58,34 @@ def test_static_scratch_entry_point_matches_the_allocating_one_twice_in_a_row():
         max_v = float(v.float().abs().max())
         assert err.max() <= MAX_ERR_FACTOR * max_v
         assert err.sum() / np.abs(want).sum() <= MRE_LIMIT
+        assert binding.regenvc_static_device_status() == 0
+        exact = oracle.cross_attention(synth.bits(q.cpu()), synth.bits(k.cpu()), synth.bits(v.cpu()))
+        assert_parity(got, exact, max_v, f"allocation-free entry point against the oracle, {n_kv} keys")
+
+
+def test_static_scratch_status_word_is_reported_and_cleared():
+    """An input beyond the fp16 operand range sets the entry point's own status word; until it is read, later
+    calls skip their work.  Reading it clears it, and the next call is normal again."""
+    L = binding.lib()
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(9001)
+    q = synth.from_f32(rng.standard_normal((300, 2, 128))).to(dev)
+    k = synth.from_f32(rng.standard_normal((140, 2, 128))).to(dev)
+    v = synth.from_f32(rng.standard_normal((140, 2, 128))).to(dev)
+    assert binding.regenvc_static_device_status() == 0
+    bad = k.clone()
+    bad[2, 0, 5] = 1e6
+    launches = binding.regenvc_kernel_launch_count()
+    assert _call_static(L, q, bad, v, torch.empty_like(q)) == binding.OK
+    assert binding.regenvc_kernel_launch_count() == launches + 2  # both launches are counted
+    assert binding.regenvc_static_device_status() == binding.ERR_RANGE
+    assert binding.regenvc_static_device_status() == 0  # cleared by the query
+    assert binding.regenvc_device_status() == 0         # the ordinary entry points' word was never touched
+    out = torch.full_like(q, float("nan"))
+    assert _call_static(L, q, k, v, out) == binding.OK
+    assert binding.regenvc_static_device_status() == 0
+    exact = oracle.cross_attention(synth.bits(q.cpu()), synth.bits(k.cpu()), synth.bits(v.cpu()))
+    assert_parity(out.double().cpu().numpy(), exact, float(v.float().abs().max()), "after the status was cleared")
 
 
 def test_static_scratch_entry_point_rejects_what_does_not_fit():
