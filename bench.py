@@ -2,14 +2,20 @@
 """Benchmark of the fused 3D-RoPE attention path on seeded synthetic tensors.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+                    [--sustain-seconds S] [--usp UxR]
 
 One "step" is one pass of the whole hot path over one window: the
 self-attention call (key/value preparation pass + attention kernel) followed by
 one cross-attention call per conditioning sequence of the workload.  At N = 1
 the workload is the 480x832 window (7x30x52 = 10920 tokens, 12 heads x 128,
 plus 512 conditioning tokens), the shape the tensor-peak target is quoted on.
-With N > 1 (one process per GPU under torchrun) every rank runs its own window
-(heads and windows are independent: no data-path collective, weak scaling).
+With N > 1 (one process per GPU under torchrun; without a launcher the script
+starts the N ranks itself) every rank runs its own window (heads and windows
+are independent: no data-path collective, weak scaling).  After the K timed
+steps the same step loop is repeated for at least S seconds (default 4) with
+the clocks sampled throughout, which gives the power-capped, sustained
+figures next to the burst ones.  --usp UxR instead spreads ONE window over
+U*R ranks as Ulysses x Ring (strong scaling, the paper's decomposition).
 
 Prints ONE JSON line on rank 0.
 """
@@ -37,7 +43,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 PAPER_CONTEXT = ("paper: 972 ms per 25-frame window (24 fps) for the WHOLE decoder on 8 consumer-class GPUs; "
                  "it reports no attention-only number")
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the self-attention kernel at the 480x832 window
-# shape, from the ncu capture summarised in profiles/attn_pipelined_kernel_window_480x832.md (101.5 MB + 18.0 MB).
+# shape, from one ncu capture of that launch (101.5 MB read + 18.0 MB written).
 ATTN_KERNEL_DRAM_TRAFFIC_BYTES = {"window_480x832": 119.4e6}
 N_BUFFER_SETS = 4
 
@@ -100,7 +106,8 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "error": self.err}
         return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
                 "reasons": sorted(self.reasons), "samples": len(self.samples),
-                "power_w_max": max(self.power) if self.power else None}
+                "power_w_max": max(self.power) if self.power else None,
+                "power_w_median": statistics.median(self.power) if self.power else None}
 
 
 def rank_seed_offset(set_index: int, rank: int) -> int:
@@ -191,22 +198,39 @@ def run_reference(args, w: synth.Workload):
 
 
 # ------------------------------------------------------------------------------------------------ CUDA path
-def run_ours(args, w: synth.Workload):
-    from paper_2607_28144_b200 import binding, build
+def _events(n):
+    return [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
 
-    build.build()
+
+def _setup_ranks(args):
+    """Rank bookkeeping.  Fails loudly when fewer ranks or GPUs than --gpus come up."""
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world != args.gpus and world > 1:
-        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torchrun --nproc-per-node {args.gpus}")
+    if torch.cuda.device_count() <= local:
+        raise SystemExit(f"rank {rank} needs cuda:{local} but only {torch.cuda.device_count()} GPU(s) are visible")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    dist = None
+    dist, seen = None, 1
     if world > 1:
         import torch.distributed as dist
 
         dist.init_process_group("nccl", device_id=dev)
+        ones = torch.ones((), dtype=torch.int32, device=dev)
+        dist.all_reduce(ones)
+        seen = int(ones.item())
+        if seen != args.gpus or dist.get_world_size() != args.gpus:
+            raise SystemExit(f"--gpus {args.gpus} but the communicator has {seen} rank(s)")
+    return rank, world, local, dev, dist, seen
+
+
+def run_ours(args, w: synth.Workload):
+    from paper_2607_28144_b200 import binding, build
+
+    build.build()
+    rank, world, local, dev, dist, ranks_seen = _setup_ranks(args)
 
     def barrier():
         if dist is not None:
@@ -221,7 +245,11 @@ def run_ours(args, w: synth.Workload):
         cross = [synth.cross_inputs(wi, n) for n in w.cross_kv]
         sets.append({"q": q.to(dev), "k": k.to(dev), "v": v.to(dev),
                      "cross": [(a.to(dev), b.to(dev)) for a, b in cross],
-                     "out": torch.empty_like(q, device=dev), "outc": [torch.empty_like(q, device=dev) for _ in cross]})
+                     "out": torch.empty_like(q, device=dev), "outc": [torch.empty_like(q, device=dev) for _ in cross],
+                     # a workspace of its own, used only where the attention kernel is timed alone: the operands
+                     # prepared from this set's k and v stay in it between launches
+                     "ws": torch.empty((binding.regenvc_workspace_bytes(w.n_tokens, w.n_heads),), dtype=torch.uint8,
+                                       device=dev)})
     host0 = None
     stream = torch.cuda.Stream(device=dev)
 
@@ -230,9 +258,47 @@ def run_ours(args, w: synth.Workload):
         for (ck, cv), oc in zip(s["cross"], s["outc"]):
             binding.regenvc_cross_attn_forward(s["q"], ck, cv, oc, stream)
 
+    def self_call(s):
+        binding.regenvc_attn_forward(s["q"], s["k"], s["v"], s["out"], w.T, w.H, w.W, w.theta, stream)
+
+    def kernel_only_loop(n, per_launch_events):
+        """n launches of the attention kernel of the self-attention call alone (operands already prepared in the
+        set's own workspace), rotating over the input sets.  Returns the per-launch times in ms, or the mean
+        over the whole loop when per_launch_events is false."""
+        binding.regenvc_debug_set_phases(2)
+        try:
+            if per_launch_events:
+                evs = _events(n)
+                for i, (a, b) in enumerate(evs):
+                    s = sets[i % N_BUFFER_SETS]
+                    binding.regenvc_set_workspace(s["ws"])
+                    a.record(stream)
+                    self_call(s)
+                    b.record(stream)
+                torch.cuda.synchronize()
+                return [a.elapsed_time(b) for a, b in evs]
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for i in range(n):
+                s = sets[i % N_BUFFER_SETS]
+                binding.regenvc_set_workspace(s["ws"])
+                self_call(s)
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / n
+        finally:
+            binding.regenvc_set_workspace(None)
+            binding.regenvc_debug_set_phases(3)
+
     with torch.cuda.stream(stream):
         for i in range(max(args.warmup, 3)):
             step(sets[i % N_BUFFER_SETS])
+        for s in sets:  # operands of every set prepared once in the set's own workspace (used by kernel_only_loop)
+            binding.regenvc_set_workspace(s["ws"])
+            self_call(s)
+        binding.regenvc_set_workspace(None)
+
+        # ---- the K timed steps of the contract
         barrier()
         sampler = ClockSampler(local)
         sampler.start()
@@ -250,30 +316,68 @@ def run_ours(args, w: synth.Workload):
         if status != 0:
             raise SystemExit(f"device status {status}: {binding.status_string(status)}")
 
-        # the dominant kernel alone: attention kernel of the self-attention call (operands already prepared)
-        s0 = sets[0]
-        step(s0)
-        binding.regenvc_attn_forward(s0["q"], s0["k"], s0["v"], s0["out"], w.T, w.H, w.W, w.theta, stream)
-        binding.regenvc_debug_set_phases(2)
+        # ---- the dominant kernel alone, burst regime: isolated launches right after a pause
+        time.sleep(0.5)
         n_k = max(10, min(args.steps, 50))
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_k)]
-        for a, b in evs:
-            a.record(stream)
-            binding.regenvc_attn_forward(s0["q"], s0["k"], s0["v"], s0["out"], w.T, w.H, w.W, w.theta, stream)
-            b.record(stream)
+        kernel_only_loop(3, True)
+        burst_sampler = ClockSampler(local)
+        burst_sampler.start()
+        attn_times = kernel_only_loop(n_k, True)
+        burst_sampler.stop()
+        attn_ms, attn_ms_best = statistics.mean(attn_times), min(attn_times)
         binding.regenvc_debug_set_phases(1)
-        evp = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_k)]
-        for a, b in evp:
+        evp = _events(n_k)
+        for i, (a, b) in enumerate(evp):
             a.record(stream)
-            binding.regenvc_attn_forward(s0["q"], s0["k"], s0["v"], s0["out"], w.T, w.H, w.W, w.theta, stream)
+            self_call(sets[i % N_BUFFER_SETS])
             b.record(stream)
         binding.regenvc_debug_set_phases(3)
         torch.cuda.synchronize()
-        attn_ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
-        attn_ms_best = min(a.elapsed_time(b) for a, b in evs)
         prep_ms = statistics.mean(a.elapsed_time(b) for a, b in evp)
 
-        # end to end through the host-buffer entry points (pinned host memory, copies inside the timed region)
+        # ---- sustained regime: the step loop repeated until at least --sustain-seconds have passed, whatever
+        # --steps is, with the clocks sampled throughout; then the attention kernel alone in the same regime
+        sustained = None
+        if args.sustain_seconds > 0:
+            chunk = max(8, int(0.05 / max(ms_total / args.steps * 1e-3, 1e-6)))  # about 50 ms of steps per event pair
+            sus_sampler = ClockSampler(local)
+            barrier()
+            sus_sampler.start()
+            t_wall0 = time.perf_counter()
+            chunks, i = [], 0
+            while True:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                for _ in range(chunk):
+                    step(sets[i % N_BUFFER_SETS])
+                    i += 1
+                b.record(stream)
+                chunks.append((a, b, time.perf_counter() - t_wall0))
+                if len(chunks) >= 2:
+                    chunks[-2][1].synchronize()  # keep one chunk queued behind the running one
+                if time.perf_counter() - t_wall0 >= args.sustain_seconds and len(chunks) >= 4:
+                    break
+            torch.cuda.synchronize()
+            t_wall = time.perf_counter() - t_wall0
+            sus_sampler.stop()
+            chunk_ms = [a.elapsed_time(b) / chunk for a, b, _ in chunks]
+            settled = [m for m, (_, _, t) in zip(chunk_ms, chunks) if t >= 0.25 * t_wall] or chunk_ms
+            # the kernel alone, still in the power-capped regime: about a second of back-to-back launches
+            ker_sampler = ClockSampler(local)
+            ker_sampler.start()
+            n_sus_k = max(50, int(1.0 / max(attn_ms * 1e-3, 1e-6)))
+            attn_ms_sus = kernel_only_loop(n_sus_k, False)
+            ker_sampler.stop()
+            sustained = {"seconds": t_wall, "steps": i, "ms_per_step": statistics.mean(settled),
+                         "ms_per_step_all": statistics.mean(chunk_ms), "ms_per_step_first_chunk": chunk_ms[0],
+                         "clocks": sus_sampler.summary(), "kernel_ms": attn_ms_sus, "kernel_launches": n_sus_k,
+                         "kernel_clocks": ker_sampler.summary()}
+            status = binding.regenvc_device_status(stream)
+            if status != 0:
+                raise SystemExit(f"device status {status}: {binding.status_string(status)}")
+
+        # ---- end to end through the host-buffer entry points (pinned host memory, copies inside the timed region)
+        s0 = sets[0]
         e2e = None
         if not args.no_e2e:
             hq, hk, hv = (t.cpu().pin_memory() for t in (s0["q"], s0["k"], s0["v"]))
@@ -290,7 +394,6 @@ def run_ours(args, w: synth.Workload):
                 host_step()
             n_e = max(3, min(args.steps, 20))
             barrier()
-            t0 = time.perf_counter()
             f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             f0.record(stream)
             for _ in range(n_e):
@@ -305,15 +408,20 @@ def run_ours(args, w: synth.Workload):
             e2e = {"ms": e2e_ms, "h2d": h2d, "d2h": d2h, "steps": n_e}
 
     # max over ranks
-    ms_total, e2e_ms, attn_ms_max = max_over_ranks([ms_total, e2e["ms"] if e2e else 0.0, attn_ms], dist, dev)
+    red = max_over_ranks([ms_total, e2e["ms"] if e2e else 0.0, attn_ms,
+                          sustained["ms_per_step"] if sustained else 0.0,
+                          sustained["kernel_ms"] if sustained else 0.0], dist, dev)
+    ms_total, e2e_ms, attn_ms_max, sus_ms, sus_kernel_ms = red
     ms_step = ms_total / args.steps
     fl = step_flops(w)
     value = whole_job_tflops(world, fl, ms_step)
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
-        peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+        burst_peak = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+        sus_peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
         achieved = w.self_flops() / (attn_ms * 1e-3) / 1e12
+        bc = burst_sampler.summary()
         line = {
             "metric": "attention bf16 TFLOP/s", "value": value, "unit": "TFLOP/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
@@ -322,23 +430,51 @@ def run_ours(args, w: synth.Workload):
             "config": {"workload": w.name, "grid_THW": [w.T, w.H, w.W], "tokens": w.n_tokens, "heads": w.n_heads,
                        "head_dim": w.head_dim, "cross_kv": list(w.cross_kv), "layers": w.layers,
                        "denoise_steps": w.steps, "parallelism": f"{world} independent window(s), one per GPU",
+                       "communicator_ranks": ranks_seen,
                        "l2": f"{N_BUFFER_SETS} rotating input sets, each {4 * w.n_tokens * w.n_heads * 256 / 1e6:.0f} MB "
                              f"of q/k/v/out (L2 is 126 MB)"},
             "ms_per_window": ms_step * w.layers * w.steps,
             "pct_of_nominal_2250": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
             "gpu_launches": int(launches),
             "clocks": sampler.summary(),
+            # the kernel timed alone (isolated launches after a pause, rotating input sets) against the burst
+            # figure of the measured cuBLAS bf16 peak: frac = achieved / peak, achieved = flops / kernel_ms_mean
             "roofline": {"bound": "tensor", "kernel": "attn_pipelined_kernel (self-attention)",
-                         "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                         "peak_source": f"{peak_kind} cuBLAS bf16 sustained (kernel timed in a back-to-back loop; "
-                                        f"fp16 and bf16 operands run at the same rate)",
-                         "frac_of_burst": achieved / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"])),
+                         "achieved": achieved, "peak": burst_peak, "unit": "TFLOP/s", "frac": achieved / burst_peak,
+                         "peak_source": f"{peak_kind} cuBLAS bf16 burst (kernel timed alone; fp16 and bf16 operands "
+                                        f"run at the same rate)",
+                         "flops_per_launch": w.self_flops(),
                          "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
-                         "kernel_ms_mean": attn_ms, "kernel_ms_best": attn_ms_best, "prep_kernel_ms": prep_ms,
+                         "kernel_ms_mean": attn_ms, "kernel_ms_best": attn_ms_best, "kernel_launches_timed": n_k,
+                         "kernel_sm_mhz_median": bc.get("sm_mhz"),
+                         "kernel_time_x_mhz": attn_ms * bc["sm_mhz"] if bc.get("sm_mhz") else None,
+                         "prep_kernel_ms": prep_ms,
                          "traffic": ATTN_KERNEL_DRAM_TRAFFIC_BYTES.get(w.name),
                          "algorithmic_hbm_bytes": 4.0 * w.n_tokens * w.n_heads * 256},
             "context": PAPER_CONTEXT,
         }
+        if sustained:
+            sc, kc = sustained["clocks"], sustained["kernel_clocks"]
+            sus_tflops = whole_job_tflops(world, fl, sus_ms)
+            sus_kernel_tflops = w.self_flops() / (sus_kernel_ms * 1e-3) / 1e12
+            line["sustained"] = {
+                "seconds": sustained["seconds"], "steps": sustained["steps"], "ms_per_step": sus_ms,
+                "ms_per_step_whole_loop": sustained["ms_per_step_all"],
+                "ms_per_step_first_chunk": sustained["ms_per_step_first_chunk"],
+                "tflops": sus_tflops, "peak": sus_peak, "frac_of_sustained_peak": sus_tflops / world / sus_peak,
+                "pct_of_nominal_2250": 100.0 * sus_tflops / world / NOMINAL_BF16_TFLOPS,
+                "ms_per_window": sus_ms * w.layers * w.steps,
+                "sm_mhz_median": sc.get("sm_mhz"), "power_w_max": sc.get("power_w_max"),
+                "power_w_median": sc.get("power_w_median"), "clock_samples": sc.get("samples"),
+                "reasons": sc.get("reasons"),
+                "time_x_mhz": sus_ms * sc["sm_mhz"] if sc.get("sm_mhz") else None,
+                "kernel": {"ms": sus_kernel_ms, "launches": sustained["kernel_launches"], "tflops": sus_kernel_tflops,
+                           "frac_of_sustained_peak": sus_kernel_tflops / sus_peak,
+                           "sm_mhz_median": kc.get("sm_mhz"), "clock_samples": kc.get("samples"),
+                           "time_x_mhz": sus_kernel_ms * kc["sm_mhz"] if kc.get("sm_mhz") else None},
+                "note": "step loop repeated for at least --sustain-seconds; ms_per_step is the mean after the "
+                        "first quarter of the loop, max over ranks",
+            }
         if e2e:
             line["e2e"] = {"value": whole_job_tflops(world, fl, e2e_ms), "unit": "TFLOP/s",
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
@@ -347,7 +483,6 @@ def run_ours(args, w: synth.Workload):
             import oracle
 
             oracle.build()
-            s0 = sets[0]
             heads = [0, w.n_heads // 2, w.n_heads - 1][: max(1, args.cpu_heads)]
             dt, flc = oracle_sample(w, heads, s0["q"].cpu(), s0["k"].cpu(), s0["v"].cpu(),
                                     [(a.cpu(), b.cpu()) for a, b in s0["cross"]])
@@ -366,6 +501,101 @@ def run_ours(args, w: synth.Workload):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------ Ulysses x Ring
+def run_usp(args, w: synth.Workload):
+    """--usp UxR: ONE window spread over U*R ranks the way the paper does it (Sec. 3.5): the token sequence is
+    sharded over the ranks, an all-to-all inside each Ulysses group turns it into a head sharding, key/value
+    blocks travel around the ring while the block-wise attention kernels run, and a second all-to-all restores
+    the sequence sharding.  Strong scaling: the work of one window is fixed.  Rank 0 checks its own output shard
+    against the oracle on sampled rows."""
+    from paper_2607_28144_b200 import binding, build, usp
+
+    build.build()
+    U, R = (int(x) for x in args.usp.lower().split("x"))
+    if U * R != args.gpus:
+        raise SystemExit(f"--usp {args.usp} needs --gpus {U * R}")
+    rank, world, local, dev, dist, ranks_seen = _setup_ranks(args)
+    layout = usp.UspLayout(world, U, R, w.n_tokens, w.n_heads)
+    pg_u = pg_r = None
+    if world > 1:
+        pg_u, pg_r = usp.make_groups(layout, rank, dist)
+    q, k, v = synth.self_inputs(w)  # every rank draws the same window and keeps its own shard
+    t0, cnt = layout.shard(rank)
+    ql, kl, vl = (x[t0:t0 + cnt].contiguous().to(dev) for x in (q, k, v))
+    attn = usp.UspAttention(layout, rank, pg_u, pg_r, ops=usp.CudaOps(), dist=dist)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    out = None
+    for _ in range(max(args.warmup, 3)):
+        out = attn(ql, kl, vl, w.T, w.H, w.W, w.theta)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = binding.regenvc_kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        out = attn(ql, kl, vl, w.T, w.H, w.W, w.theta)
+    e1.record()
+    barrier()
+    sampler.stop()
+    launches = binding.regenvc_kernel_launch_count() - launches0
+    status = binding.regenvc_device_status()
+    if status != 0:
+        raise SystemExit(f"device status {status}: {binding.status_string(status)}")
+    (ms_total,) = max_over_ranks([e0.elapsed_time(e1)], dist, dev)
+    ms_step = ms_total / args.steps
+    if rank == 0:
+        line = {
+            "metric": "attention bf16 TFLOP/s", "value": w.self_flops() / (ms_step * 1e-3) / 1e12, "unit": "TFLOP/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "fp16 operands (from bf16), fp32 accumulate, bf16 out", "data": "synthetic",
+            "config": {"workload": w.name, "grid_THW": [w.T, w.H, w.W], "tokens": w.n_tokens, "heads": w.n_heads,
+                       "head_dim": w.head_dim, "parallelism": f"one window over Ulysses {U} x Ring {R}",
+                       "communicator_ranks": ranks_seen, "tokens_per_rank": cnt, "heads_per_rank": w.n_heads // U,
+                       "note": "self-attention only; inputs and outputs stay sequence-sharded on the ranks"},
+            "gpu_launches": int(launches), "clocks": sampler.summary(), "context": PAPER_CONTEXT,
+        }
+        if not args.no_cpu_baseline:
+            import oracle
+
+            oracle.build()
+            rows = np.unique(np.concatenate([np.arange(min(4, cnt)), np.linspace(0, cnt - 1, num=min(24, cnt)).astype(np.int64)]))
+            got = out.cpu()
+            qb, kb, vb = synth.bits(q), synth.bits(k), synth.bits(v)
+            num = den = 0.0
+            for head in sorted({0, w.n_heads // 2, w.n_heads - 1}):
+                ref = oracle.self_attn_head(qb, kb, vb, w.T, w.H, w.W, head, w.theta, rows=(rows + t0))
+                num += float(np.abs(got[rows, head].double().numpy() - ref).sum())
+                den += float(np.abs(ref).sum())
+            line["shard_check_mre"] = num / den
+            if num / den > 2e-3:
+                raise SystemExit(f"rank 0's output shard disagrees with the oracle: mre {num / den}")
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def respawn_under_torchrun(args):
+    """`python bench.py --gpus N` with N > 1 and no launcher: start the N ranks ourselves (one process per GPU,
+    rendezvous on 127.0.0.1) by re-executing this command line under torch.distributed.run."""
+    import socket
+
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    os.execv(sys.executable, cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -373,13 +603,24 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="window_480x832", choices=synth.WORKLOAD_ORDER)
+    ap.add_argument("--usp", default=None, metavar="UxR",
+                    help="spread ONE window over U*R = --gpus ranks as Ulysses x Ring (the paper's decomposition)")
+    ap.add_argument("--sustain-seconds", type=float, default=4.0,
+                    help="length of the sustained leg (the step loop repeated under the power cap); 0 skips it")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-heads", type=int, default=3)
     args = ap.parse_args()
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be at least 1")
     w = synth.WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, w)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        respawn_under_torchrun(args)
+    if args.usp:
+        run_usp(args, w)
     else:
         run_ours(args, w)
 

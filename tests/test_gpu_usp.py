@@ -141,6 +141,106 @@ def test_usp_paper_degrees_on_a_window_slice():
         assert_parity(got[rows, a].double().numpy(), ref, float(v.float().abs().max()), f"usp 4x2 head {a}")
 
 
+class _ThreadFabric:
+    """In-process stand-in for the process-group calls UspAttention makes, for ranks that run as host THREADS on
+    one GPU: messages are device tensors handed over through FIFO queues per (source, destination).  All waiting
+    happens on the host, never inside a kernel, and every rank's kernels go to the same stream."""
+
+    def __init__(self, world):
+        import queue
+        self.q = {(s, d): queue.Queue() for s in range(world) for d in range(world)}
+
+    def endpoint(self, rank):
+        return _ThreadDist(self, rank)
+
+
+class _ThreadDist:
+    isend, irecv = "isend", "irecv"
+
+    class _Req:
+        def __init__(self, fn):
+            self.fn = fn
+
+        def wait(self):
+            self.fn()
+
+    def __init__(self, fabric, rank):
+        self.f, self.rank = fabric, rank
+
+    def all_to_all_single(self, recv, send, output_split_sizes, input_split_sizes, group):
+        at = 0
+        for peer, n in zip(group, input_split_sizes):
+            self.f.q[(self.rank, peer)].put(send[at:at + n].clone())
+            at += n
+        assert at == send.shape[0]
+        at = 0
+        for peer, n in zip(group, output_split_sizes):
+            msg = self.f.q[(peer, self.rank)].get(timeout=120)
+            assert msg.shape[0] == n
+            recv[at:at + n].copy_(msg)
+            at += n
+        assert at == recv.shape[0]
+
+    def P2POp(self, op, tensor, peer, group):
+        return (op, tensor, peer)
+
+    def batch_isend_irecv(self, ops):
+        reqs = []
+        for op, tensor, peer in ops:
+            if op == self.isend:
+                self.f.q[(self.rank, peer)].put(tensor.clone())
+                reqs.append(self._Req(lambda: None))
+            else:
+                reqs.append(self._Req(lambda t=tensor, p=peer: t.copy_(self.f.q[(p, self.rank)].get(timeout=120))))
+        return reqs
+
+
+@pytest.mark.parametrize("grid,h,U,R", [((2, 9, 14), 4, 1, 1), ((2, 9, 14), 4, 2, 1), ((3, 10, 13), 2, 1, 2),
+                                        ((2, 16, 20), 8, 2, 2), ((2, 12, 26), 12, 4, 2)])
+def test_per_rank_driver_with_the_cuda_kernels_on_host_threads(grid, h, U, R):
+    """usp.UspAttention with usp.CudaOps -- the per-rank driver exactly as a multi-GPU job runs it: packing by the
+    resharding kernels, exchange, block-wise attention, merge, exchange back -- for every rank of a U x R layout,
+    each rank a host thread on this one GPU.  Only the transport under all_to_all_single / batch_isend_irecv is
+    replaced (queues of device tensors instead of NCCL); the joined output shards must equal unsharded attention."""
+    import threading
+
+    T, H, W = grid
+    N, world = T * H * W, U * R
+    rng = np.random.default_rng(8100 + N + 10 * U + R)
+    q = synth.from_f32(rng.standard_normal((N, h, D)))
+    k = synth.from_f32(rng.standard_normal((N, h, D)) * 1.5)
+    v = synth.from_f32(rng.standard_normal((N, h, D)))
+    dev = torch.device("cuda:0")
+    layout = usp.UspLayout(world, U, R, N, h)
+    fabric = _ThreadFabric(world)
+    outs, errs = [None] * world, []
+
+    def run(rank):
+        try:
+            torch.cuda.set_device(dev)
+            t0, cnt = layout.shard(rank)
+            ql, kl, vl = (x[t0:t0 + cnt].contiguous().to(dev) for x in (q, k, v))
+            attn = usp.UspAttention(layout, rank, layout.ulysses_group(rank), layout.ring_group(rank),
+                                    ops=usp.CudaOps(), dist=fabric.endpoint(rank))
+            outs[rank] = attn(ql, kl, vl, T, H, W).cpu()
+        except Exception as ex:  # surfaced below: a dead thread would leave its peers waiting on their queues
+            errs.append((rank, repr(ex)))
+
+    threads = [threading.Thread(target=run, args=(g,)) for g in range(world)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=300)
+    assert not errs, errs
+    assert all(o is not None for o in outs)
+    assert binding.regenvc_device_status() == 0
+    got = torch.cat(outs)
+    ref = oracle.self_attention(synth.bits(q), synth.bits(k), synth.bits(v), T, H, W)
+    assert_parity(f64(got), ref, float(v.float().abs().max()), f"per-rank driver U={U} R={R}")
+    emu = torch.cat(usp.usp_attention_one_gpu(q.to(dev), k.to(dev), v.to(dev), T, H, W, layout)).cpu()
+    assert torch.equal(got, emu)  # same kernels on the same data in the same order as the one-thread emulation
+
+
 def test_resharding_bandwidth_report(capsys):
     """HBM-bound copies: prints the achieved rate at the 480x832 window shape (run with -s to see it) and checks
     that it is at least a sizeable fraction of the memory system's (a regression guard, not a tuning target)."""

@@ -56,3 +56,25 @@ def test_two_gloo_ranks_agree_on_max_time_and_run_distinct_windows():
     w = synth.WORKLOADS["tiny"]
     assert out[0]["value"] == pytest.approx(2 * bench.step_flops(w) / 15e-3 / 1e12)
     assert bench.max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
+
+
+def test_bench_starts_its_own_ranks_and_fails_loudly_without_enough_gpus():
+    """`python bench.py --gpus 2` without a launcher re-executes itself under torch.distributed.run (two ranks,
+    rendezvous on 127.0.0.1).  On a machine with fewer than two GPUs every rank must stop with a clear message
+    instead of quietly measuring one GPU."""
+    import subprocess
+
+    if torch.cuda.device_count() >= 2:
+        pytest.skip("two GPUs are present: the command would run the benchmark itself")
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1", "--warmup", "1"],
+                       env=env, cwd=ROOT, capture_output=True, text=True, timeout=600)
+    text = r.stdout + r.stderr
+    assert r.returncode != 0
+    assert "rank 1 needs cuda:1" in text
+    assert '"n_gpus"' not in r.stdout  # no result line
+    # a rank count that contradicts --gpus is refused as well
+    env2 = dict(env, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"],
+                       env=env2, cwd=ROOT, capture_output=True, text=True, timeout=600)
+    assert r.returncode != 0 and "WORLD_SIZE=1" in (r.stdout + r.stderr)
