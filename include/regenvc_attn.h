@@ -21,9 +21,10 @@
  *     Scores are scaled by 1/sqrt(head_dim).  No mask.
  *   - Arithmetic: inputs are widened exactly; rotated Q/K, V and the softmax
  *     probabilities are rounded to fp16 tensor-core operands (inputs must
- *     therefore be finite with |x| <= 65504); all accumulation is fp32; the
- *     output is rounded once to bf16 (nearest even).  NaN/Inf inputs give
- *     unspecified results.
+ *     therefore be finite with |x| <= 65504); where nothing is rotated
+ *     (cross-attention) Q and K enter Q.K^T as the bf16 values they are; all
+ *     accumulation is fp32; the output is rounded once to bf16 (nearest
+ *     even).  NaN/Inf inputs give unspecified results.
  *   - Pointers marked "device" must be valid on the current CUDA device and
  *     16-byte aligned; the caller owns them, and the library neither frees
  *     nor keeps them beyond the stream-ordered work of the call.
@@ -89,6 +90,37 @@ int regenvc_attn_forward(const void* q, const void* k, const void* v, void* out,
  */
 int regenvc_cross_attn_forward(const void* q, const void* k, const void* v, void* out,
                                int n_q, int n_kv, int n_heads, int head_dim, void* stream);
+
+/*
+ * Conditioning keys/values prepared once (Sec. 3.9: the text and image conditioning key/value tensors are
+ * computed once per sequence and reused by every block, step and window).  regenvc_cross_attn_forward()
+ * rewrites k and v into tensor-core operand form on every call; these three calls split that off:
+ *
+ * regenvc_prepared_bytes(): size of the operand buffer for n_kv keys (0 for invalid arguments):
+ *   K' : 16-bit [n_heads][n_kv_pad][128], then V't : fp16 [n_heads][128][n_kv_pad], n_kv_pad = n_kv rounded up
+ *   to a multiple of 128, padding zero.
+ * regenvc_cross_kv_prepare(): fills `prepared` (device, caller-owned, 256-byte aligned, at least
+ *   regenvc_prepared_bytes() bytes, not overlapping k or v) from k, v [n_kv, n_heads, head_dim] bf16.  K' keeps
+ *   the bf16 bits of k; V't is v converted to fp16 and transposed.  An element of v beyond the fp16 range sets
+ *   the sticky REGENVC_ERR_RANGE status.
+ * regenvc_cross_attn_forward_prepared(): regenvc_cross_attn_forward() on a buffer filled by the call above
+ *   (same n_kv and n_heads); bit-identical result, one kernel instead of two.  `prepared` is only read, so
+ *   calls on different streams may share it; the thread's workspace is still used for split-key scratch.
+ *
+ * regenvc_attn_forward_prepared(): attention on operands a producer has already written in operand form
+ *   (a fused QKV-projection epilogue: regenvc_qkv_rope_project()):
+ *   q_rot    : device, fp16 [n_q, n_heads, 128], rotated queries
+ *   prepared : K' fp16 (rotated keys) and V't fp16 in the layout above; the padding columns of V't must be finite
+ *   out      : device, bf16 [n_q, n_heads, 128]
+ *   No rotation, conversion or preparation pass happens inside the call.
+ */
+size_t regenvc_prepared_bytes(int n_kv, int n_heads, int head_dim);
+int regenvc_cross_kv_prepare(const void* k, const void* v, void* prepared,
+                             int n_kv, int n_heads, int head_dim, void* stream);
+int regenvc_cross_attn_forward_prepared(const void* q, const void* prepared, void* out,
+                                        int n_q, int n_kv, int n_heads, int head_dim, void* stream);
+int regenvc_attn_forward_prepared(const void* q_rot, const void* prepared, void* out,
+                                  int n_q, int n_kv, int n_heads, int head_dim, void* stream);
 
 /*
  * Block-wise attention for sequence-parallel use (Sec. 3.5: Ring attention streams key/value blocks around
@@ -203,7 +235,7 @@ int regenvc_static_device_status(void* stream, int* status_out);
 /*
  * Scratch memory.  Each call first rewrites the keys and values into
  * tensor-core operand form in a device workspace:
- *   K' : fp16 [n_heads][n_kv_pad][128]   rotated (self) or converted (cross) keys
+ *   K' : 16-bit [n_heads][n_kv_pad][128] rotated fp16 keys (self) or the bf16 keys as they are (cross)
  *   V't: fp16 [n_heads][128][n_kv_pad]   values, transposed so that keys are contiguous
  * with n_kv_pad = n_kv rounded up to a multiple of 128 (padding is zero),
  * K' first, V't directly after it, followed by a fixed 21,299,200-byte area

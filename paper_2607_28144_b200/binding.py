@@ -24,7 +24,9 @@ EXPORTS = [
     "regenvc_cross_attn_forward_host", "regenvc_workspace_bytes", "regenvc_set_workspace",
     "regenvc_device_status", "regenvc_status_string", "regenvc_last_cuda_error", "regenvc_version",
     "regenvc_kernel_launch_count", "regenvc_shutdown", "regenvc_debug_set_phases",
-    "regenvc_cross_attn_forward_static", "regenvc_static_device_status", "regenvc_attn_partial", "regenvc_attn_merge",
+    "regenvc_cross_attn_forward_static", "regenvc_static_device_status", "regenvc_attn_partial",
+    "regenvc_prepared_bytes", "regenvc_cross_kv_prepare", "regenvc_cross_attn_forward_prepared",
+    "regenvc_attn_forward_prepared", "regenvc_attn_merge",
     "regenvc_ulysses_scatter_heads", "regenvc_ulysses_gather_heads", "regenvc_debug_expire_wait",
 ]
 
@@ -66,6 +68,14 @@ def lib() -> ctypes.CDLL:
     L.regenvc_attn_forward_host.restype = i32
     L.regenvc_cross_attn_forward_host.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
     L.regenvc_cross_attn_forward_host.restype = i32
+    L.regenvc_prepared_bytes.argtypes = [i32, i32, i32]
+    L.regenvc_prepared_bytes.restype = sz
+    L.regenvc_cross_kv_prepare.argtypes = [vp, vp, vp, i32, i32, i32, vp]
+    L.regenvc_cross_kv_prepare.restype = i32
+    L.regenvc_cross_attn_forward_prepared.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
+    L.regenvc_cross_attn_forward_prepared.restype = i32
+    L.regenvc_attn_forward_prepared.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
+    L.regenvc_attn_forward_prepared.restype = i32
     L.regenvc_workspace_bytes.argtypes = [i32, i32, i32]
     L.regenvc_workspace_bytes.restype = sz
     L.regenvc_set_workspace.argtypes = [vp, sz]
@@ -142,6 +152,56 @@ def regenvc_cross_attn_forward(q, k, v, out, stream=None):
         raise ValueError("shape mismatch")
     _check(lib().regenvc_cross_attn_forward(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), n_q, n_kv, h, d,
                                             _stream(stream)))
+    return out
+
+
+def regenvc_prepared_bytes(n_kv: int, n_heads: int, head_dim: int = 128) -> int:
+    return int(lib().regenvc_prepared_bytes(n_kv, n_heads, head_dim))
+
+
+def regenvc_cross_kv_prepare(k, v, prepared=None, stream=None):
+    """Rewrites conditioning keys/values [n_kv, h, d] into operand form once; returns the ``prepared`` buffer
+    (a CUDA uint8 tensor, allocated here with torch when not given) for regenvc_cross_attn_forward_prepared."""
+    for t, nm in ((k, "k"), (v, "v")):
+        _dev_bf16(t, nm)
+    n_kv, h, d = k.shape
+    if v.shape != k.shape:
+        raise ValueError("shape mismatch")
+    need = regenvc_prepared_bytes(n_kv, h, d)
+    if prepared is None:
+        prepared = torch.empty((need,), dtype=torch.uint8, device=k.device)
+    if prepared.dtype != torch.uint8 or not prepared.is_cuda or prepared.numel() < need:
+        raise TypeError(f"prepared must be a CUDA uint8 tensor of at least {need} bytes")
+    _check(lib().regenvc_cross_kv_prepare(k.data_ptr(), v.data_ptr(), prepared.data_ptr(), n_kv, h, d, _stream(stream)))
+    return prepared
+
+
+def regenvc_cross_attn_forward_prepared(q, prepared, n_kv: int, out, stream=None):
+    """Cross-attention of q [n_q, h, d] to the n_kv conditioning tokens whose operands are in ``prepared``."""
+    _dev_bf16(q, "q")
+    _dev_bf16(out, "out")
+    n_q, h, d = q.shape
+    if out.shape != q.shape:
+        raise ValueError("shape mismatch")
+    if prepared.dtype != torch.uint8 or not prepared.is_cuda or prepared.numel() < regenvc_prepared_bytes(n_kv, h, d):
+        raise TypeError("prepared is too small for this shape")
+    _check(lib().regenvc_cross_attn_forward_prepared(q.data_ptr(), prepared.data_ptr(), out.data_ptr(), n_q, n_kv, h, d,
+                                                     _stream(stream)))
+    return out
+
+
+def regenvc_attn_forward_prepared(q_rot, prepared, n_kv: int, out, stream=None):
+    """Attention on operands already in operand form: q_rot fp16 [n_q, h, d] (rotated), ``prepared`` = K' and V't."""
+    if q_rot.dtype != torch.float16 or not q_rot.is_cuda or not q_rot.is_contiguous() or q_rot.dim() != 3:
+        raise TypeError("q_rot must be a contiguous CUDA fp16 tensor [tokens, heads, head_dim]")
+    _dev_bf16(out, "out")
+    n_q, h, d = q_rot.shape
+    if out.shape != q_rot.shape:
+        raise ValueError("shape mismatch")
+    if prepared.dtype != torch.uint8 or not prepared.is_cuda or prepared.numel() < regenvc_prepared_bytes(n_kv, h, d):
+        raise TypeError("prepared is too small for this shape")
+    _check(lib().regenvc_attn_forward_prepared(q_rot.data_ptr(), prepared.data_ptr(), out.data_ptr(), n_q, n_kv, h, d,
+                                               _stream(stream)))
     return out
 
 

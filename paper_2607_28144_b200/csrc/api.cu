@@ -230,6 +230,13 @@ struct BlockArgs {
     float* tok_o = nullptr;
     float2* tok_ml = nullptr;
     int phases = -1;  // bit 0: preparation pass, bit 1: attention; -1: the calling thread's debug setting
+    // Caller-owned operand buffer (K' then V't, regenvc_prepared_bytes()): the preparation pass writes it and the
+    // attention kernel reads it instead of the workspace, which then only serves the split-key scratch.
+    void* prepared = nullptr;
+    // q is a 16-bit tensor already in operand form (rotated where that applies, same type as K'): the kernel's
+    // TMA warp copies the query tiles; qk_bf16 says whether that type is bf16 (else fp16).
+    bool q_operand = false;
+    bool qk_bf16 = false;
 };
 
 int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int n_kv, int n_heads, bool rope, int T,
@@ -240,7 +247,8 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     int rc = device_state(&dev, &st);
     if (rc != REGENVC_OK) return rc;
 
-    const size_t need = workspace_need(n_kv, n_heads);
+    const int phases = blk.phases >= 0 ? blk.phases : tl_phases;
+    const size_t need = !blk.prepared ? workspace_need(n_kv, n_heads) : ((phases & 2) ? kSplitScratchBytes : 0);
     void* ws = nullptr;
     Workspace* own = nullptr;  // the library's workspace of this thread, when the caller supplied none
     if (tl_user_ws.ptr) {
@@ -255,8 +263,12 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
         if (rc != REGENVC_OK) return rc;
     }
     const int kv_pad = round_up(n_kv, kTile);
-    __half* kp = reinterpret_cast<__half*>(ws);
+    __half* kp = reinterpret_cast<__half*>(blk.prepared ? blk.prepared : ws);
     __half* vt = kp + (size_t)n_heads * kv_pad * kHeadDim;
+    // Without rotation the queries need no arithmetic before Q.K^T: both they and the keys stay bf16 (their
+    // products are then exact) and the query tiles are copied by TMA straight from the caller's tensor.
+    const bool q_operand = blk.q_operand || !rope;
+    const bool qk_bf16 = blk.q_operand ? blk.qk_bf16 : !rope;
 
     RopeGrid grid{nullptr, T, H, W};
     if (rope) {
@@ -265,7 +277,8 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     }
 
     CUtensorMap tmap_k, tmap_v;
-    rc = make_tmap(&tmap_k, kp, kHeadDim, (uint64_t)n_heads * kv_pad, kHeadDim * sizeof(__half));
+    rc = make_tmap(&tmap_k, kp, kHeadDim, (uint64_t)n_heads * kv_pad, kHeadDim * sizeof(__half),
+                   qk_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
     if (rc != REGENVC_OK) return rc;
     rc = make_tmap(&tmap_v, vt, (uint64_t)kv_pad, (uint64_t)n_heads * kHeadDim, (uint64_t)kv_pad * sizeof(__half));
     if (rc != REGENVC_OK) return rc;
@@ -279,10 +292,10 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     pp.n_kv_pad = kv_pad;
     pp.h = n_heads;
     pp.rope = rope ? 1 : 0;
+    pp.k_bf16 = qk_bf16 ? 1 : 0;
     pp.grid = grid;
     pp.pos_offset = blk.kv_token0;
     pp.status = st->status;
-    const int phases = blk.phases >= 0 ? blk.phases : tl_phases;
     if (phases & 1) {
         CUDA_TRY(launch_prep_kv(pp, stream));
         launched();
@@ -297,6 +310,7 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     ap.n_kv_pad = kv_pad;
     ap.h = n_heads;
     ap.rope = rope ? 1 : 0;
+    ap.qk_bf16 = qk_bf16 ? 1 : 0;
     ap.grid = grid;
     ap.q_pos_offset = blk.q_token0;
     ap.tok_o = blk.tok_o;
@@ -312,7 +326,7 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     ap.n_full_items = n_items;
     ap.split_k = 1;
     ap.tiles_per_piece = n_tiles;
-    ap.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + operand_bytes(n_kv, n_heads));
+    ap.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + (blk.prepared ? 0 : operand_bytes(n_kv, n_heads)));
     ap.part_ml = reinterpret_cast<float2*>(ap.part_o + (size_t)kMaxPieceCtas * 2 * kTile * kHeadDim);
     const int rem = n_items % st->sm_count;
     if (rem > 0 && st->sm_count <= kMaxPieceCtas && blk.tok_o == nullptr) {
@@ -330,7 +344,14 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     rc = make_tmap(&tmap_out, out != nullptr ? out : const_cast<void*>(q), (uint64_t)n_heads * kHeadDim, (uint64_t)n_q,
                    (uint64_t)n_heads * kHeadDim * sizeof(__nv_bfloat16), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     if (rc != REGENVC_OK) return rc;
-    CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, ap, stream));
+    CUtensorMap tmap_q;
+    if (q_operand) {
+        rc = make_tmap(&tmap_q, const_cast<void*>(q), (uint64_t)n_heads * kHeadDim, (uint64_t)n_q,
+                       (uint64_t)n_heads * kHeadDim * 2,
+                       qk_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
+        if (rc != REGENVC_OK) return rc;
+    }
+    CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, stream));
     launched();
     if (ap.split_k > 1) {
         MergeParams mp;
@@ -472,6 +493,69 @@ int regenvc_cross_attn_forward(const void* q, const void* k, const void* v, void
     int rc = validate(q, k, v, out, n_q, n_kv, n_heads, head_dim, true);
     if (rc != REGENVC_OK) return rc;
     return enqueue(q, k, v, out, n_q, n_kv, n_heads, false, 1, 1, 1, 1.0f, (cudaStream_t)stream);
+}
+
+size_t regenvc_prepared_bytes(int n_kv, int n_heads, int head_dim) {
+    if (n_kv < 1 || n_heads < 1 || head_dim != kHeadDim) return 0;
+    return operand_bytes(n_kv, n_heads);
+}
+
+int regenvc_cross_kv_prepare(const void* k, const void* v, void* prepared, int n_kv, int n_heads, int head_dim,
+                             void* stream) {
+    // the ordinary checks with a one-row stand-in for q/out: `prepared` must not overlap k or v
+    if (!k || !v || !prepared) return REGENVC_ERR_NULL_POINTER;
+    if (n_kv < 1 || n_heads < 1 || head_dim < 1) return REGENVC_ERR_BAD_SHAPE;
+    const long long kv_pad = ((long long)n_kv + kTile - 1) / kTile * kTile;
+    if (n_kv > (1 << 30) || n_heads > 65535 || kv_pad * n_heads >= (1ll << 31)) return REGENVC_ERR_BAD_SHAPE;
+    if (head_dim != kHeadDim) return REGENVC_ERR_UNSUPPORTED;
+    if (((uintptr_t)k | (uintptr_t)v) & 15) return REGENVC_ERR_MISALIGNED;
+    if ((uintptr_t)prepared & 255) return REGENVC_ERR_MISALIGNED;
+    const size_t kb = (size_t)n_kv * n_heads * kHeadDim * 2, pb = operand_bytes(n_kv, n_heads);
+    if (overlaps(prepared, pb, k, kb) || overlaps(prepared, pb, v, kb)) return REGENVC_ERR_ALIASING;
+    BlockArgs blk;
+    blk.phases = 1;
+    blk.prepared = prepared;
+    return enqueue(nullptr, k, v, nullptr, 1, n_kv, n_heads, false, 1, 1, 1, 1.0f, (cudaStream_t)stream, blk);
+}
+
+namespace {
+// Checks shared by the two calls that run attention on operands prepared earlier.
+int validate_prepared(const void* q, const void* prepared, void* out, int n_q, int n_kv, int n_heads, int head_dim) {
+    if (!q || !prepared || !out) return REGENVC_ERR_NULL_POINTER;
+    if (n_q < 1 || n_kv < 1 || n_heads < 1 || head_dim < 1) return REGENVC_ERR_BAD_SHAPE;
+    const long long kv_pad = ((long long)n_kv + kTile - 1) / kTile * kTile;
+    if (n_q > (1 << 30) || n_kv > (1 << 30) || n_heads > 65535 || kv_pad * n_heads >= (1ll << 31) ||
+        (long long)n_q * n_heads >= (1ll << 31))
+        return REGENVC_ERR_BAD_SHAPE;
+    if (head_dim != kHeadDim) return REGENVC_ERR_UNSUPPORTED;
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return REGENVC_ERR_MISALIGNED;
+    if ((uintptr_t)prepared & 255) return REGENVC_ERR_MISALIGNED;
+    const size_t qb = (size_t)n_q * n_heads * kHeadDim * 2, pb = operand_bytes(n_kv, n_heads);
+    if (overlaps(out, qb, q, qb) || overlaps(out, qb, prepared, pb)) return REGENVC_ERR_ALIASING;
+    return REGENVC_OK;
+}
+}  // namespace
+
+int regenvc_cross_attn_forward_prepared(const void* q, const void* prepared, void* out, int n_q, int n_kv,
+                                        int n_heads, int head_dim, void* stream) {
+    int rc = validate_prepared(q, prepared, out, n_q, n_kv, n_heads, head_dim);
+    if (rc != REGENVC_OK) return rc;
+    BlockArgs blk;
+    blk.phases = 2;
+    blk.prepared = const_cast<void*>(prepared);
+    return enqueue(q, nullptr, nullptr, out, n_q, n_kv, n_heads, false, 1, 1, 1, 1.0f, (cudaStream_t)stream, blk);
+}
+
+int regenvc_attn_forward_prepared(const void* q_rot, const void* prepared, void* out, int n_q, int n_kv, int n_heads,
+                                  int head_dim, void* stream) {
+    int rc = validate_prepared(q_rot, prepared, out, n_q, n_kv, n_heads, head_dim);
+    if (rc != REGENVC_OK) return rc;
+    BlockArgs blk;
+    blk.phases = 2;
+    blk.prepared = const_cast<void*>(prepared);
+    blk.q_operand = true;   // fp16 queries, rotated by whoever produced them
+    blk.qk_bf16 = false;
+    return enqueue(q_rot, nullptr, nullptr, out, n_q, n_kv, n_heads, false, 1, 1, 1, 1.0f, (cudaStream_t)stream, blk);
 }
 
 int regenvc_attn_forward_host(const void* q, const void* k, const void* v, void* out, int T, int H, int W, int n_heads,

@@ -56,7 +56,8 @@ constexpr int kMmaWarp = kSoftmaxThreads / 32, kTmaWarp = kMmaWarp + 1;
 #endif
 // bit i set: pair i of every eight probability pairs takes the polynomial 2^x instead of the MUFU
 constexpr uint32_t kPolyMask = REGENVC_POLY_MASK;
-constexpr uint32_t kIdesc = umma_idesc_f16_f32acc(128, 128);
+constexpr uint32_t kIdesc = umma_idesc_f16_f32acc(128, 128);           // fp16 x fp16 -> fp32
+constexpr uint32_t kIdescBf16 = umma_idesc_bf16_f32acc(128, 128);      // bf16 x bf16 -> fp32
 constexpr uint32_t kSmemBytes = (2 + kStages) * kTileBytes + 1024 /*align*/ + 256 /*barriers*/ + 8192 /*row exchange*/;
 constexpr uint64_t kWaitLimitNs = 500000000ull;   // 0.5 s per wait
 
@@ -178,12 +179,12 @@ __device__ __forceinline__ void exp_chunk(const uint32_t* s, uint64_t scale2, ui
 
 // The eight K = 16 steps of one 128 x 128 x 128 product.  Descriptors differ only in the start-address
 // field: +2 (32 bytes) per K step inside a 128-byte row, +1024 (16 KB) for the second 64-element block.
-__device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint32_t sQ, uint32_t sK) {
+__device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint32_t sQ, uint32_t sK, uint32_t idesc) {
     const uint64_t a0 = umma_smem_desc_k_sw128(sQ), b0 = umma_smem_desc_k_sw128(sK);
 #pragma unroll
     for (int kk = 0; kk < 8; ++kk) {
         const uint64_t off = (kk >> 2) * (kBlockBytes >> 4) + (kk & 3) * 2;
-        umma_ss(d_tmem, a0 + off, b0 + off, kIdesc, kk > 0);
+        umma_ss(d_tmem, a0 + off, b0 + off, idesc, kk > 0);
     }
 }
 __device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint32_t sV, bool accumulate) {
@@ -200,9 +201,14 @@ __device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint3
 
 }  // namespace
 
+// kQTma = false: the softmax warps fetch the bf16 query rows, rotate them and write the fp16 tiles themselves.
+// kQTma = true : the query tiles are already in operand form in global memory (16-bit, same type as K', token-major)
+//                and the TMA warp copies them; the softmax warps go straight to the first score tile.
+template <bool kQTma>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
-                      const __grid_constant__ CUtensorMap tmap_out, const AttnParams p) {
+                      const __grid_constant__ CUtensorMap tmap_out, const __grid_constant__ CUtensorMap tmap_q,
+                      const AttnParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = base;                       // 2 tiles
@@ -238,7 +244,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             mbar_init(smem_u32(&bar->kv_empty[s]), 1);
         }
         for (int t = 0; t < 2; ++t) {
-            mbar_init(smem_u32(&bar->q_full[t]), kSoftmaxThreads);
+            mbar_init(smem_u32(&bar->q_full[t]), kQTma ? 1 : kSoftmaxThreads);
             mbar_init(smem_u32(&bar->s_full[t]), 1);
             mbar_init(smem_u32(&bar->p_full[t]), kSoftmaxThreads);
             mbar_init(smem_u32(&bar->o_full[t]), 1);
@@ -256,6 +262,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         tma_prefetch_desc(&tmap_k);
         tma_prefetch_desc(&tmap_v);
         tma_prefetch_desc(&tmap_out);
+        if (kQTma) tma_prefetch_desc(&tmap_q);
       }
       __syncwarp();
       tc_fence_before();
@@ -266,6 +273,16 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
       if (warp == kTmaWarp) {
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
+            if (kQTma) {
+                // rows past n_q lie outside the tensor map and arrive as zeros
+                for (int t = 0; t < (tile1_active ? 2 : 1); ++t) {
+                    const uint32_t full = smem_u32(&bar->q_full[t]);
+                    const uint32_t dst = smem_u32(sQ + t * kTileBytes);
+                    mbar_expect_tx(full, kTileBytes);
+                    tma_load_2d(dst, &tmap_q, head * kHeadDim, q0 + t * kTile, full);
+                    tma_load_2d(dst + kBlockBytes, &tmap_q, head * kHeadDim + 64, q0 + t * kTile, full);
+                }
+            }
             const int total = 2 * n_tiles;
             for (int i = 0; i < total; ++i) {
                 const int slot = i % kStages, round = i / kStages;
@@ -288,13 +305,14 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         if (elect_one()) {
             const uint32_t sQ0 = smem_u32(sQ), sQ1 = smem_u32(sQ) + kTileBytes;
             const int n_active = tile1_active ? 2 : 1;
+            const uint32_t idesc_qk = p.qk_bf16 ? kIdescBf16 : kIdesc;
             bool ok = mbar_wait(smem_u32(&bar->q_full[0]), 0, ctl);
             if (ok && tile1_active) ok = mbar_wait(smem_u32(&bar->q_full[1]), 0, ctl);
             if (ok) ok = mbar_wait(smem_u32(&bar->kv_full[0]), 0, ctl);
             if (ok) {
                 tc_fence_after();
                 for (int t = 0; t < n_active; ++t) {
-                    issue_qk(tmem_base + t * 128, t ? sQ1 : sQ0, smem_u32(sKV));
+                    issue_qk(tmem_base + t * 128, t ? sQ1 : sQ0, smem_u32(sKV), idesc_qk);
                     umma_commit(smem_u32(&bar->s_full[t]));
                 }
                 umma_commit(smem_u32(&bar->kv_empty[0]));
@@ -312,7 +330,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     issue_pv(tmem_base + 256 + t * 128, tmem_base + t * 128, smem_u32(sKV + slot_v * kTileBytes), j > 0);
                     umma_commit(smem_u32(&bar->o_full[t]));
                     if (more) {
-                        issue_qk(tmem_base + t * 128, t ? sQ1 : sQ0, smem_u32(sKV + slot_k * kTileBytes));
+                        issue_qk(tmem_base + t * 128, t ? sQ1 : sQ0, smem_u32(sKV + slot_k * kTileBytes), idesc_qk);
                         umma_commit(smem_u32(&bar->s_full[t]));
                     }
                 }
@@ -329,13 +347,16 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         const int part = warp >> 2;                      // which kColsPerThread key columns of a score row
         const int row = (warp & 3) * 32 + lane;          // row in the tile == TMEM lane
         const int n_active = tile1_active ? 2 : 1;
-        if (tile1_active) load_rotate_q_tiles<kSoftmaxThreads, 2>(p, head, q0, sQ, tid);
-        else load_rotate_q_tiles<kSoftmaxThreads, 1>(p, head, q0, sQ, tid);
-        fence_proxy_async_smem();
+        if (!kQTma) {
+            if (tile1_active) load_rotate_q_tiles<kSoftmaxThreads, 2>(p, head, q0, sQ, tid);
+            else load_rotate_q_tiles<kSoftmaxThreads, 1>(p, head, q0, sQ, tid);
+            fence_proxy_async_smem();
+        }
         setup_done_wait();   // barriers and tensor memory exist from here on
         tc_fence_after();
         tmem_base = bar->tmem_base;
-        for (int t = 0; t < n_active; ++t) mbar_arrive(smem_u32(&bar->q_full[t]));
+        if (!kQTma)
+            for (int t = 0; t < n_active; ++t) mbar_arrive(smem_u32(&bar->q_full[t]));
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         const float scale = p.scale_log2;
         const uint64_t scale2 = pack2(scale, scale);
@@ -535,20 +556,32 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
 }
 
 
-cudaError_t configure_attn_pipelined() {
+namespace {
+template <bool kQTma>
+cudaError_t configure_one() {
     cudaFuncAttributes attr;
-    cudaError_t e = cudaFuncGetAttributes(&attr, attn_pipelined_kernel);
+    cudaError_t e = cudaFuncGetAttributes(&attr, attn_pipelined_kernel<kQTma>);
     if (e != cudaSuccess) return e;
     // the register hand-over above assumes the kernel was compiled to exactly kLaunchRegs registers per thread
     if (attr.numRegs != kLaunchRegs) return cudaErrorInvalidConfiguration;
-    return cudaFuncSetAttribute(attn_pipelined_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    return cudaFuncSetAttribute(attn_pipelined_kernel<kQTma>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)kSmemBytes);
+}
+}  // namespace
+
+cudaError_t configure_attn_pipelined() {
+    cudaError_t e = configure_one<false>();
+    return e != cudaSuccess ? e : configure_one<true>();
 }
 
 cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
-                                  const AttnParams& p, cudaStream_t stream) {
+                                  const CUtensorMap* tmap_q, const AttnParams& p, cudaStream_t stream) {
     const int n_items = p.pairs_per_head * p.h;
     dim3 grid(p.n_full_items + (n_items - p.n_full_items) * p.split_k);
-    attn_pipelined_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmap_k, tmap_v, tmap_out, p);
+    if (tmap_q)
+        attn_pipelined_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(tmap_k, tmap_v, tmap_out, *tmap_q, p);
+    else
+        attn_pipelined_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(tmap_k, tmap_v, tmap_out, tmap_out, p);
     return cudaGetLastError();
 }
 

@@ -34,6 +34,7 @@ struct PrepParams {
     __half* vt;               // [h][128][n_kv_pad]
     int n_kv, n_kv_pad, h;
     int rope;                 // 1: rotate k by the 3D rotary embedding
+    int k_bf16;               // 1: K' keeps the bf16 bits of k (no rotation, no conversion); 0: fp16
     RopeGrid grid;
     int pos_offset;           // token index (in the T x H x W grid) of row 0 of k
     int* status;
@@ -44,6 +45,7 @@ struct AttnParams {
     __nv_bfloat16* out;       // [n_q, h, 128]
     int n_q, n_kv, n_kv_pad, h;
     int rope;
+    int qk_bf16;              // 1: the query tiles and K' are bf16 (Q.K^T runs bf16 x bf16), 0: fp16
     RopeGrid grid;
     float scale_log2;         // log2(e) / sqrt(head_dim)
     int* status;
@@ -112,8 +114,10 @@ int record_cuda_failure(cudaError_t e, const char* what);
 
 // Launchers (each returns the launch error, enqueues on `stream`).
 cudaError_t launch_prep_kv(const PrepParams& p, cudaStream_t stream);
+// tmap_q != nullptr: the query tiles are copied by TMA from a 16-bit tensor already in operand form (same type as
+// K'); nullptr: the kernel reads p.q (bf16), rotates if p.rope and converts to fp16 itself.
 cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
-                                  const AttnParams& p, cudaStream_t stream);
+                                  const CUtensorMap* tmap_q, const AttnParams& p, cudaStream_t stream);
 cudaError_t configure_attn_pipelined();   // once per device: register hand-over check, large dynamic shared memory
 cudaError_t launch_merge_partials(const MergeParams& p, cudaStream_t stream);
 cudaError_t launch_merge_token_partials(const TokenMergeParams& p, cudaStream_t stream);

@@ -1,7 +1,8 @@
 // Key/value preparation pass: one read of K and V, one write of the two
 // tensor-core operand tensors the attention kernel streams through TMA.
 //   K' [h][n_kv_pad][128] fp16 : keys, rotated by the 3D rotary embedding
-//                                (self-attention) or just converted (cross)
+//                                (self-attention) or just converted (cross);
+//                                with k_bf16 set the bf16 bits are kept as they are
 //   V't [h][128][n_kv_pad] fp16: values transposed so that keys are the
 //                                contiguous (K-major) dimension of P.V
 // Rotating K here, once per key, replaces rotating every K tile again in each
@@ -49,6 +50,10 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
         for (int it = 0; it < kTile / 16; ++it) {
             const int row = it * 16 + (tid >> 4);
             const int n = tile0 + row;
+            if (p.k_bf16) {  // uniform over the grid: the keys stay bf16 (cross-attention with bf16 queries)
+                reinterpret_cast<uint4*>(p.kp + ((size_t)head * p.n_kv_pad + n) * kHeadDim)[chunk] = raw[it];
+                continue;
+            }
             float x[8];
             bf16x8_to_float(raw[it], x);
             if (p.rope && n < p.n_kv) rope_rotate8(x, p.grid, s_pos[row], rc);

@@ -108,8 +108,9 @@ extern "C" int regenvc_cross_attn_forward_static(const void* q, const void* k, c
 
     __half* kp = reinterpret_cast<__half*>(dev->scratch);
     __half* vt = kp + (size_t)n_heads * kv_pad * kHeadDim;
-    CUtensorMap tmap_k, tmap_v, tmap_out;
-    rc = encode_map(&tmap_k, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, kp, kHeadDim, (uint64_t)n_heads * kv_pad,
+    // as in regenvc_cross_attn_forward(): queries and keys stay bf16, the query tiles are copied by TMA
+    CUtensorMap tmap_k, tmap_v, tmap_out, tmap_q;
+    rc = encode_map(&tmap_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, kp, kHeadDim, (uint64_t)n_heads * kv_pad,
                     kHeadDim * sizeof(__half));
     if (rc == REGENVC_OK)
         rc = encode_map(&tmap_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, vt, (uint64_t)kv_pad, (uint64_t)n_heads * kHeadDim,
@@ -117,6 +118,9 @@ extern "C" int regenvc_cross_attn_forward_static(const void* q, const void* k, c
     if (rc == REGENVC_OK)
         rc = encode_map(&tmap_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, out, (uint64_t)n_heads * kHeadDim, (uint64_t)n_q,
                         (uint64_t)n_heads * kHeadDim * sizeof(__nv_bfloat16));
+    if (rc == REGENVC_OK)
+        rc = encode_map(&tmap_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, const_cast<void*>(q), (uint64_t)n_heads * kHeadDim,
+                        (uint64_t)n_q, (uint64_t)n_heads * kHeadDim * sizeof(__nv_bfloat16));
     if (rc != REGENVC_OK) return rc;
 
     PrepParams pp;
@@ -128,6 +132,7 @@ extern "C" int regenvc_cross_attn_forward_static(const void* q, const void* k, c
     pp.n_kv_pad = (int)kv_pad;
     pp.h = n_heads;
     pp.rope = 0;
+    pp.k_bf16 = 1;
     pp.grid = RopeGrid{nullptr, 1, 1, 1};
     pp.pos_offset = 0;
     pp.status = dev->status;
@@ -143,6 +148,7 @@ extern "C" int regenvc_cross_attn_forward_static(const void* q, const void* k, c
     ap.n_kv_pad = (int)kv_pad;
     ap.h = n_heads;
     ap.rope = 0;
+    ap.qk_bf16 = 1;
     ap.grid = pp.grid;
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)kHeadDim));
     ap.status = dev->status;
@@ -156,7 +162,7 @@ extern "C" int regenvc_cross_attn_forward_static(const void* q, const void* k, c
     ap.tok_ml = nullptr;
     ap.part_o = nullptr;
     ap.part_ml = nullptr;
-    e = launch_attn_pipelined(tmap_k, tmap_v, tmap_out, ap, (cudaStream_t)stream);
+    e = launch_attn_pipelined(tmap_k, tmap_v, tmap_out, &tmap_q, ap, (cudaStream_t)stream);
     if (e != cudaSuccess) return record_cuda_failure(e, "launch of the attention kernel");
     count_launch();
     return REGENVC_OK;

@@ -13,6 +13,11 @@ __host__ __device__ constexpr uint32_t umma_idesc_f16_f32acc(int m, int n) {
            (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
 
+// The same with both operands bf16 (format code 1 in the A and B fields).
+__host__ __device__ constexpr uint32_t umma_idesc_bf16_f32acc(int m, int n) {
+    return umma_idesc_f16_f32acc(m, n) | (1u << 7) | (1u << 10);
+}
+
 // 64-bit shared-memory matrix descriptor for a K-major operand stored as
 // rows of 128 bytes (64 16-bit elements) with the 128-byte swizzle, eight
 // rows per 1024-byte group (the layout a TMA box of {64, rows} with

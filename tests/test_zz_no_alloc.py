@@ -73,10 +73,10 @@ def test_static_scratch_status_word_is_reported_and_cleared():
     k = synth.from_f32(rng.standard_normal((140, 2, 128))).to(dev)
     v = synth.from_f32(rng.standard_normal((140, 2, 128))).to(dev)
     assert binding.regenvc_static_device_status() == 0
-    bad = k.clone()
-    bad[2, 0, 5] = 1e6
+    bad = v.clone()
+    bad[2, 0, 5] = 1e6  # a value beyond the fp16 range (keys stay bf16 here and have no such limit)
     launches = binding.regenvc_kernel_launch_count()
-    assert _call_static(L, q, bad, v, torch.empty_like(q)) == binding.OK
+    assert _call_static(L, q, k, bad, torch.empty_like(q)) == binding.OK
     assert binding.regenvc_kernel_launch_count() == launches + 2  # both launches are counted
     assert binding.regenvc_static_device_status() == binding.ERR_RANGE
     assert binding.regenvc_static_device_status() == 0  # cleared by the query
