@@ -15,6 +15,7 @@ from .oracle import (  # noqa: F401
     rope_angle,
     rope_freq,
     rope_pair,
+    rope_rotate_f64,
     rope_rotate_head,
     rope_split,
     self_attention,
@@ -22,3 +23,4 @@ from .oracle import (  # noqa: F401
     threads,
     token_position,
 )
+from . import qkv_oracle  # noqa: E402,F401

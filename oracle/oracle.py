@@ -60,6 +60,8 @@ def _load():
     L.oracle_rope_angle.restype = f64
     L.oracle_rope_rotate_head.argtypes = [p, p, i32, i32, i32, i32, i32, i32, f64, i32]
     L.oracle_rope_rotate_head.restype = i32
+    L.oracle_rope_rotate_f64.argtypes = [p, p, i32, i32, i32, i32, f64]
+    L.oracle_rope_rotate_f64.restype = i32
     L.oracle_widen_head.argtypes = [p, p, i64, i32, i32, i32]
     L.oracle_widen_head.restype = i32
     L.oracle_attn_core_head.argtypes = [p, p, p, i64, i64, i32, p, i64, p]
@@ -129,6 +131,16 @@ def rope_rotate_head(x, T, H, W, head, theta=10000.0, pairing=PAIR_ADJACENT) -> 
     out = np.empty((N, d), dtype=np.float64)
     _check(_load().oracle_rope_rotate_head(_ptr(x), _ptr(out), T, H, W, h, d, head, float(theta), pairing),
            "rope_rotate_head")
+    return out
+
+
+def rope_rotate_f64(x, T, H, W, theta=10000.0) -> np.ndarray:
+    """Rotation of one head's fp64 vectors [T*H*W, d] (adjacent pairs)."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    N, d = x.shape
+    assert N == T * H * W
+    out = np.empty_like(x)
+    _check(_load().oracle_rope_rotate_f64(_ptr(x), _ptr(out), T, H, W, d, float(theta)), "rope_rotate_f64")
     return out
 
 

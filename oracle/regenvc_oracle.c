@@ -146,6 +146,26 @@ int oracle_rope_rotate_head(const uint16_t *in, double *out, int T, int H, int W
     return ORACLE_OK;
 }
 
+/* The same rotation for vectors that are already fp64 (one head, [n_tokens, d]): used where the
+ * rotated tensor is produced by an earlier fp64 step instead of being read as bf16. */
+int oracle_rope_rotate_f64(const double *in, double *out, int T, int H, int W, int d, double theta)
+{
+    if (!in || !out || T < 1 || H < 1 || W < 1 || d < 2 || (d & 1) || !(theta > 0.0))
+        return ORACLE_BAD_ARG;
+    int64_t N = (int64_t)T * H * W;
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+        for (int j = 0; j < d / 2; ++j) {
+            double phi = oracle_rope_angle(n, j, H, W, d, theta);
+            double c = cos(phi), s = sin(phi);
+            double a = in[(size_t)n * d + 2 * j], b = in[(size_t)n * d + 2 * j + 1];
+            out[(size_t)n * d + 2 * j] = a * c - b * s;
+            out[(size_t)n * d + 2 * j + 1] = a * s + b * c;
+        }
+    }
+    return ORACLE_OK;
+}
+
 /* Widen one head without rotation: bf16 [n_tokens, h, d] -> fp64 [n_tokens, d]. */
 int oracle_widen_head(const uint16_t *in, double *out, int64_t n_tokens, int h, int d, int head)
 {
