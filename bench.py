@@ -226,6 +226,57 @@ def _setup_ranks(args):
     return rank, world, local, dev, dist, seen
 
 
+def time_producer_fusion(binding, w: synth.Workload, dev, stream, n=20):
+    """Times, with CUDA events on `stream`, (a) the fused producer + attention on its operands and (b) the same
+    block computed as projection-then-attention with library kernels in front of the ordinary call."""
+    C, N, h = w.n_heads * w.head_dim, w.n_tokens, w.n_heads
+    x, wq, b, gq, gk, eps = (t.to(dev) if torch.is_tensor(t) else t for t in synth.block_inputs(w))
+    q_rot, prepared = binding.regenvc_qkv_rope_project(x, wq, b, gq, gk, eps, w.T, w.H, w.W, h, w.theta, stream=stream)
+    out = torch.empty((N, h, w.head_dim), dtype=torch.bfloat16, device=dev)
+    b16 = b.to(torch.bfloat16)
+
+    def producer():
+        binding.regenvc_qkv_rope_project(x, wq, b, gq, gk, eps, w.T, w.H, w.W, h, w.theta, q_rot=q_rot,
+                                         prepared=prepared, stream=stream)
+
+    def attn_prepared():
+        binding.regenvc_attn_forward_prepared(q_rot, prepared, N, out, stream)
+
+    def library_projection():
+        y = torch.addmm(b16, x, wq.t()).float()
+        q, k = y[:, :C], y[:, C:2 * C]
+        q = (q * torch.rsqrt(q.pow(2).mean(-1, keepdim=True) + eps) * gq).to(torch.bfloat16).view(N, h, w.head_dim)
+        k = (k * torch.rsqrt(k.pow(2).mean(-1, keepdim=True) + eps) * gk).to(torch.bfloat16).view(N, h, w.head_dim)
+        return q, k, y[:, 2 * C:].to(torch.bfloat16).view(N, h, w.head_dim)
+
+    q, k, v = (t.contiguous() for t in library_projection())
+
+    def attn_plain():
+        binding.regenvc_attn_forward(q, k, v, out, w.T, w.H, w.W, w.theta, stream)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        evs = _events(n)
+        for a, bb in evs:
+            a.record(stream)
+            fn()
+            bb.record(stream)
+        torch.cuda.synchronize()
+        return statistics.mean(a.elapsed_time(bb) for a, bb in evs)
+
+    t_prod, t_attn_p = timed(producer), timed(attn_prepared)
+    t_gemm = timed(lambda: torch.addmm(b16, x, wq.t()))
+    t_lib, t_attn = timed(library_projection), timed(attn_plain)
+    flops = 2.0 * N * 3 * C * C
+    return {"producer_ms": t_prod, "producer_tflops": flops / (t_prod * 1e-3) / 1e12,
+            "attention_on_prepared_operands_ms": t_attn_p, "fused_ms": t_prod + t_attn_p,
+            "library_gemm_only_ms": t_gemm, "library_projection_norm_ms": t_lib,
+            "attention_with_preparation_pass_ms": t_attn, "unfused_ms": t_lib + t_attn,
+            "note": "fused = regenvc_qkv_rope_project + regenvc_attn_forward_prepared (no preparation pass, no "
+                    "bf16 round trip of q, k, v); unfused = library GEMM + eager norm kernels + regenvc_attn_forward"}
+
+
 def run_ours(args, w: synth.Workload):
     from paper_2607_28144_b200 import binding, build
 
@@ -376,6 +427,13 @@ def run_ours(args, w: synth.Workload):
             if status != 0:
                 raise SystemExit(f"device status {status}: {binding.status_string(status)}")
 
+        # ---- producer fusion: the block's QKV projection with norm, rotation and operand layout fused into its
+        # epilogue, followed by attention on those operands, against projection-then-attention (library GEMM and
+        # element-wise kernels writing bf16 q, k, v, then the ordinary self-attention call)
+        fusion = None
+        if not args.no_producer and w.n_heads % 2 == 0 and w.n_heads <= 16:
+            fusion = time_producer_fusion(binding, w, dev, stream)
+
         # ---- end to end through the host-buffer entry points (pinned host memory, copies inside the timed region)
         s0 = sets[0]
         e2e = None
@@ -475,6 +533,8 @@ def run_ours(args, w: synth.Workload):
                 "note": "step loop repeated for at least --sustain-seconds; ms_per_step is the mean after the "
                         "first quarter of the loop, max over ranks",
             }
+        if fusion:
+            line["producer_fusion"] = fusion
         if e2e:
             line["e2e"] = {"value": whole_job_tflops(world, fl, e2e_ms), "unit": "TFLOP/s",
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
@@ -608,6 +668,7 @@ def main():
     ap.add_argument("--sustain-seconds", type=float, default=4.0,
                     help="length of the sustained leg (the step loop repeated under the power cap); 0 skips it")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-producer", action="store_true", help="skip the producer-fusion leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-heads", type=int, default=3)
     args = ap.parse_args()

@@ -123,6 +123,36 @@ int regenvc_attn_forward_prepared(const void* q_rot, const void* prepared, void*
                                   int n_q, int n_kv, int n_heads, int head_dim, void* stream);
 
 /*
+ * Producer fusion: the QKV projection of a transformer block with the steps between it and the attention
+ * kernel fused into its epilogue.  The paper takes the backbone by reference (Sec. 3.2, 3.4); in that block
+ *     y_q = x W_q^T + b_q,  y_k = x W_k^T + b_k,  v = x W_v^T + b_v,
+ *     q = y_q * g_q / sqrt(mean_c y_q[c]^2 + eps)   (RMS norm over ALL n_heads * 128 features of a token), k alike,
+ * heads are consecutive blocks of 128 features, and q, k are then rotated by the 3D rotary embedding.  This call
+ * computes all of it in one pass and writes the results directly in the operand form
+ * regenvc_attn_forward_prepared() consumes, so that neither a preparation pass nor a bf16 round trip of q, k, v
+ * exists on this path:
+ *   x        : device, bf16 [T*H*W, C], C = n_heads * 128                     (read only)
+ *   w_qkv    : device, bf16 [3C, C]; row f = weights of output feature f; rows 0..C-1 q, C..2C-1 k, 2C..3C-1 v
+ *   b_qkv    : device, fp32 [3C], or NULL for no bias
+ *   g_q, g_k : device, fp32 [C] norm gains, or NULL for ones;  eps >= 0
+ *   q_rot    : device, fp16 [T*H*W, n_heads, 128]                              (written)
+ *   prepared : device, 256-byte aligned, regenvc_prepared_bytes(T*H*W, n_heads, 128) bytes: K' then V't (written,
+ *              padding zero)
+ * Arithmetic: bf16 products accumulated in fp32, norm and rotation in fp32, one rounding to fp16.  A result
+ * beyond the fp16 range sets the sticky REGENVC_ERR_RANGE status.  n_heads must be even and at most 16 (the
+ * n_heads / 2 thread blocks that share a token tile exchange their partial sums of squares as one cluster):
+ * otherwise REGENVC_ERR_UNSUPPORTED.  Asynchronous on `stream`; allocates only the rotary table of a new
+ * (T, H, W, theta).  Typical use:
+ *     regenvc_qkv_rope_project(x, w, b, gq, gk, eps, q_rot, prepared, T, H, W, h, 128, theta, s);
+ *     regenvc_attn_forward_prepared(q_rot, prepared, out, T*H*W, T*H*W, h, 128, s);
+ */
+int regenvc_qkv_rope_project(const void* x, const void* w_qkv, const void* b_qkv,
+                             const void* g_q, const void* g_k, float eps,
+                             void* q_rot, void* prepared,
+                             int T, int H, int W, int n_heads, int head_dim,
+                             float rope_theta, void* stream);
+
+/*
  * Block-wise attention for sequence-parallel use (Sec. 3.5: Ring attention streams key/value blocks around
  * the devices and combines the per-block results by the online-softmax rule; the result is unsharded
  * attention, only summed in another order).

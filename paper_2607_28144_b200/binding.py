@@ -26,7 +26,7 @@ EXPORTS = [
     "regenvc_kernel_launch_count", "regenvc_shutdown", "regenvc_debug_set_phases",
     "regenvc_cross_attn_forward_static", "regenvc_static_device_status", "regenvc_attn_partial",
     "regenvc_prepared_bytes", "regenvc_cross_kv_prepare", "regenvc_cross_attn_forward_prepared",
-    "regenvc_attn_forward_prepared", "regenvc_attn_merge",
+    "regenvc_attn_forward_prepared", "regenvc_qkv_rope_project", "regenvc_attn_merge",
     "regenvc_ulysses_scatter_heads", "regenvc_ulysses_gather_heads", "regenvc_debug_expire_wait",
 ]
 
@@ -76,6 +76,8 @@ def lib() -> ctypes.CDLL:
     L.regenvc_cross_attn_forward_prepared.restype = i32
     L.regenvc_attn_forward_prepared.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
     L.regenvc_attn_forward_prepared.restype = i32
+    L.regenvc_qkv_rope_project.argtypes = [vp, vp, vp, vp, vp, f32, vp, vp, i32, i32, i32, i32, i32, f32, vp]
+    L.regenvc_qkv_rope_project.restype = i32
     L.regenvc_workspace_bytes.argtypes = [i32, i32, i32]
     L.regenvc_workspace_bytes.restype = sz
     L.regenvc_set_workspace.argtypes = [vp, sz]
@@ -203,6 +205,37 @@ def regenvc_attn_forward_prepared(q_rot, prepared, n_kv: int, out, stream=None):
     _check(lib().regenvc_attn_forward_prepared(q_rot.data_ptr(), prepared.data_ptr(), out.data_ptr(), n_q, n_kv, h, d,
                                                _stream(stream)))
     return out
+
+
+def regenvc_qkv_rope_project(x, w_qkv, b_qkv, g_q, g_k, eps: float, T: int, H: int, W: int, n_heads: int,
+                             rope_theta: float = 10000.0, q_rot=None, prepared=None, stream=None):
+    """QKV projection with fused RMS norm, rotation and operand layout.  x: CUDA bf16 [T*H*W, C]; w_qkv: CUDA bf16
+    [3C, C]; b_qkv (fp32 [3C]), g_q, g_k (fp32 [C]) may be None.  Returns (q_rot fp16 [N, h, 128], prepared uint8),
+    allocated here with torch when not given; feed them to regenvc_attn_forward_prepared."""
+    if x.dtype != torch.bfloat16 or not x.is_cuda or not x.is_contiguous() or x.dim() != 2:
+        raise TypeError("x must be a contiguous CUDA bf16 tensor [tokens, C]")
+    n, C = x.shape
+    if n != T * H * W or C != n_heads * 128:
+        raise ValueError("x must be [T*H*W, n_heads * 128]")
+    if w_qkv.dtype != torch.bfloat16 or not w_qkv.is_cuda or not w_qkv.is_contiguous() or tuple(w_qkv.shape) != (3 * C, C):
+        raise TypeError("w_qkv must be a contiguous CUDA bf16 tensor [3C, C]")
+    for t, nm, size in ((b_qkv, "b_qkv", 3 * C), (g_q, "g_q", C), (g_k, "g_k", C)):
+        if t is not None and (t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous() or t.numel() != size):
+            raise TypeError(f"{nm} must be a contiguous CUDA fp32 tensor of {size} elements (or None)")
+    if q_rot is None:
+        q_rot = torch.empty((n, n_heads, 128), dtype=torch.float16, device=x.device)
+    need = regenvc_prepared_bytes(n, n_heads, 128)
+    if prepared is None:
+        prepared = torch.empty((need,), dtype=torch.uint8, device=x.device)
+    if q_rot.dtype != torch.float16 or tuple(q_rot.shape) != (n, n_heads, 128) or not q_rot.is_contiguous():
+        raise TypeError("q_rot must be a contiguous CUDA fp16 tensor [tokens, heads, 128]")
+    if prepared.dtype != torch.uint8 or prepared.numel() < need:
+        raise TypeError(f"prepared must be a CUDA uint8 tensor of at least {need} bytes")
+    ptr = lambda t: None if t is None else t.data_ptr()  # noqa: E731
+    _check(lib().regenvc_qkv_rope_project(x.data_ptr(), w_qkv.data_ptr(), ptr(b_qkv), ptr(g_q), ptr(g_k), float(eps),
+                                          q_rot.data_ptr(), prepared.data_ptr(), T, H, W, n_heads, 128,
+                                          float(rope_theta), _stream(stream)))
+    return q_rot, prepared
 
 
 def regenvc_cross_attn_forward_static(q, k, v, out, stream=None):

@@ -123,6 +123,7 @@ int device_state(int* dev_out, DeviceState** st_out) {
                 g_encode = (EncodeTiledFn)fn;
             }
             CUDA_TRY(configure_attn_pipelined());
+            CUDA_TRY(configure_qkv_project());
             CUDA_TRY(cudaMalloc(&st.status, sizeof(int)));
             CUDA_TRY(cudaMemset(st.status, 0, sizeof(int)));
         }
@@ -201,10 +202,10 @@ int rope_table(DeviceState& st, int T, int H, int W, float theta, const float2**
 }
 
 int make_tmap(CUtensorMap* m, void* base, uint64_t inner, uint64_t outer, uint64_t row_bytes,
-              CUtensorMapDataType type = CU_TENSOR_MAP_DATA_TYPE_FLOAT16) {
+              CUtensorMapDataType type = CU_TENSOR_MAP_DATA_TYPE_FLOAT16, uint32_t box_rows = 128) {
     const cuuint64_t gdim[2] = {inner, outer};
     const cuuint64_t gstride[1] = {row_bytes};
-    const cuuint32_t box[2] = {64, 128};
+    const cuuint32_t box[2] = {64, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode(m, type, 2, base, gdim, gstride, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -556,6 +557,64 @@ int regenvc_attn_forward_prepared(const void* q_rot, const void* prepared, void*
     blk.q_operand = true;   // fp16 queries, rotated by whoever produced them
     blk.qk_bf16 = false;
     return enqueue(q_rot, nullptr, nullptr, out, n_q, n_kv, n_heads, false, 1, 1, 1, 1.0f, (cudaStream_t)stream, blk);
+}
+
+int regenvc_qkv_rope_project(const void* x, const void* w_qkv, const void* b_qkv, const void* g_q, const void* g_k,
+                             float eps, void* q_rot, void* prepared, int T, int H, int W, int n_heads, int head_dim,
+                             float rope_theta, void* stream) {
+    if (!x || !w_qkv || !q_rot || !prepared) return REGENVC_ERR_NULL_POINTER;
+    long long n = 0;
+    int rc = check_self_args(T, H, W, rope_theta, &n);
+    if (rc != REGENVC_OK) return rc;
+    if (n_heads < 1 || head_dim < 1) return REGENVC_ERR_BAD_SHAPE;
+    const long long n_pad = (n + kTile - 1) / kTile * kTile;
+    if (n_heads > 65535 || n_pad * n_heads >= (1ll << 31)) return REGENVC_ERR_BAD_SHAPE;
+    if (head_dim != kHeadDim || n_heads % kProjHeadsPerCta != 0 || n_heads / kProjHeadsPerCta > kProjMaxCluster)
+        return REGENVC_ERR_UNSUPPORTED;
+    if (!(rope_theta > 0.0f) || !std::isfinite(rope_theta) || !(eps >= 0.0f) || !std::isfinite(eps))
+        return REGENVC_ERR_UNSUPPORTED;
+    if (((uintptr_t)x | (uintptr_t)w_qkv | (uintptr_t)q_rot | (uintptr_t)b_qkv | (uintptr_t)g_q | (uintptr_t)g_k) & 15)
+        return REGENVC_ERR_MISALIGNED;
+    if ((uintptr_t)prepared & 255) return REGENVC_ERR_MISALIGNED;
+    const size_t C = (size_t)n_heads * kHeadDim;
+    const size_t xb = (size_t)n * C * 2, wb = 3 * C * C * 2, pb = operand_bytes(n, n_heads);
+    if (overlaps(q_rot, xb, x, xb) || overlaps(q_rot, xb, w_qkv, wb) || overlaps(prepared, pb, x, xb) ||
+        overlaps(prepared, pb, w_qkv, wb) || overlaps(prepared, pb, q_rot, xb))
+        return REGENVC_ERR_ALIASING;
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev = 0;
+    DeviceState* st = nullptr;
+    rc = device_state(&dev, &st);
+    if (rc != REGENVC_OK) return rc;
+    ProjParams pp;
+    pp.bias = reinterpret_cast<const float*>(b_qkv);
+    pp.g_q = reinterpret_cast<const float*>(g_q);
+    pp.g_k = reinterpret_cast<const float*>(g_k);
+    pp.eps = eps;
+    pp.n_tokens = (int)n;
+    pp.n_pad = (int)n_pad;
+    pp.C = (int)C;
+    pp.h = n_heads;
+    pp.grid = RopeGrid{nullptr, T, H, W};
+    pp.status = st->status;
+    rc = rope_table(*st, T, H, W, rope_theta, &pp.grid.tab);
+    if (rc != REGENVC_OK) return rc;
+    __half* kp = reinterpret_cast<__half*>(prepared);
+    __half* vt = kp + (size_t)n_heads * n_pad * kHeadDim;
+    CUtensorMap tmap_x, tmap_w, tmap_q, tmap_k, tmap_v;
+    rc = make_tmap(&tmap_x, const_cast<void*>(x), C, (uint64_t)n, C * 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
+    if (rc == REGENVC_OK)
+        rc = make_tmap(&tmap_w, const_cast<void*>(w_qkv), C, 3 * C, C * 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                       kProjHeadsPerCta * kHeadDim);
+    if (rc == REGENVC_OK) rc = make_tmap(&tmap_q, q_rot, C, (uint64_t)n, C * 2);
+    if (rc == REGENVC_OK) rc = make_tmap(&tmap_k, kp, kHeadDim, (uint64_t)n_heads * n_pad, kHeadDim * sizeof(__half));
+    if (rc == REGENVC_OK)
+        rc = make_tmap(&tmap_v, vt, (uint64_t)n_pad, (uint64_t)n_heads * kHeadDim, (uint64_t)n_pad * sizeof(__half));
+    if (rc != REGENVC_OK) return rc;
+    CUDA_TRY(launch_qkv_project(tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, pp, (cudaStream_t)stream));
+    launched();
+    return REGENVC_OK;
 }
 
 int regenvc_attn_forward_host(const void* q, const void* k, const void* v, void* out, int T, int H, int W, int n_heads,

@@ -67,6 +67,23 @@ struct AttnParams {
     float2* part_ml;          // [piece CTA][256 rows] (reference m in log2 units, row sum l)
 };
 
+// QKV projection with fused norm / rotation / operand-layout epilogue (producer of the attention operands).
+constexpr int kProjHeadsPerCta = 2;   // a CTA computes 128 tokens x two heads of one of q, k, v
+constexpr int kProjMaxCluster = 8;    // the CTAs that share a token tile form one cluster (h / 2 of them)
+struct ProjParams {
+    const float* bias;        // [3C] or nullptr
+    const float* g_q;         // [C] RMS-norm gains of q (nullptr: ones)
+    const float* g_k;         // [C]
+    float eps;
+    int n_tokens, n_pad, C, h;
+    RopeGrid grid;
+    int* status;
+};
+cudaError_t configure_qkv_project();
+cudaError_t launch_qkv_project(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w, const CUtensorMap& tmap_q,
+                               const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const ProjParams& p,
+                               cudaStream_t stream);
+
 // Merge of token-major partial results of several key/value blocks.
 constexpr int kMaxMergeParts = 8;
 struct TokenMergeParams {

@@ -23,7 +23,7 @@ HEAD_DIM = 128
 ROPE_THETA = 10000.0
 
 # generator streams
-STREAM_Q, STREAM_K, STREAM_V, STREAM_CK, STREAM_CV, STREAM_SCALE = range(6)
+STREAM_Q, STREAM_K, STREAM_V, STREAM_CK, STREAM_CV, STREAM_SCALE, STREAM_X, STREAM_W, STREAM_B, STREAM_G = range(10)
 
 
 @dataclass(frozen=True)
@@ -96,6 +96,19 @@ def cross_inputs(w: Workload, n_kv: int):
     k = normal_bf16(w.seed + 1000 * n_kv, STREAM_CK, n_kv, w.n_heads, w.head_dim)
     v = normal_bf16(w.seed + 1000 * n_kv, STREAM_CV, n_kv, w.n_heads, w.head_dim)
     return k, v
+
+
+def block_inputs(w: Workload):
+    """Inputs of the producer step in front of self-attention (the block's QKV projection): token features
+    x [N, C] ~ N(0, 1) bf16, weights w_qkv [3C, C] ~ N(0, 1/C) bf16 (so that projected features are O(1), as after a
+    normalisation layer), bias [3C] ~ N(0, 0.1^2) fp32, norm gains g_q, g_k [C] ~ U[0.5, 1.5] fp32, eps = 1e-6.
+    Stand-ins for activations and trained weights, which are not available here."""
+    C = w.n_heads * w.head_dim
+    x = torch.randn((w.n_tokens, C), generator=_gen(w.seed, STREAM_X), dtype=torch.float32).to(torch.bfloat16)
+    wq = (torch.randn((3 * C, C), generator=_gen(w.seed, STREAM_W), dtype=torch.float32) / C ** 0.5).to(torch.bfloat16)
+    b = 0.1 * torch.randn((3 * C,), generator=_gen(w.seed, STREAM_B), dtype=torch.float32)
+    g = 0.5 + torch.rand((2, C), generator=_gen(w.seed, STREAM_G), dtype=torch.float32)
+    return x, wq, b, g[0].contiguous(), g[1].contiguous(), 1e-6
 
 
 def bits(t: torch.Tensor) -> np.ndarray:
