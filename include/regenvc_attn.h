@@ -296,8 +296,11 @@ int regenvc_device_status(void* stream, int* status_out);
  * thread enqueue.  Bit 0 = key/value preparation pass, bit 1 = attention
  * kernel; the default is 3 (both).  With bit 0 clear the workspace must still
  * hold the prepared operands of the same k, v and shape (from an earlier full
- * call), which lets a benchmark time the attention kernel alone.  Returns
- * REGENVC_ERR_BAD_SHAPE for a mask outside 1..3.
+ * call), which lets a benchmark time the attention kernel alone.  Bit 2 (value
+ * 4, together with bit 0 and/or 1) makes calls with short key sequences use
+ * one thread block per work item instead of the persistent form they
+ * normally take (same results; for measuring the difference).  Returns
+ * REGENVC_ERR_BAD_SHAPE for a mask outside 1..7 or without bit 0 and bit 1.
  */
 int regenvc_debug_set_phases(int mask);
 

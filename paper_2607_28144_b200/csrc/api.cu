@@ -124,6 +124,7 @@ int device_state(int* dev_out, DeviceState** st_out) {
             }
             CUDA_TRY(configure_attn_pipelined());
             CUDA_TRY(configure_qkv_project());
+            CUDA_TRY(configure_attn_persistent());
             CUDA_TRY(cudaMalloc(&st.status, sizeof(int)));
             CUDA_TRY(cudaMemset(st.status, 0, sizeof(int)));
         }
@@ -329,8 +330,11 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     ap.tiles_per_piece = n_tiles;
     ap.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + (blk.prepared ? 0 : operand_bytes(n_kv, n_heads)));
     ap.part_ml = reinterpret_cast<float2*>(ap.part_o + (size_t)kMaxPieceCtas * 2 * kTile * kHeadDim);
+    // Short key sequences with query tiles in operand form: one persistent CTA per SM walks over the items and
+    // overlaps their fixed costs (no key-range pieces in that form).
+    const bool persistent = q_operand && blk.tok_o == nullptr && n_tiles <= kPersistentMaxTiles && !(tl_phases & 4);
     const int rem = n_items % st->sm_count;
-    if (rem > 0 && st->sm_count <= kMaxPieceCtas && blk.tok_o == nullptr) {
+    if (!persistent && rem > 0 && st->sm_count <= kMaxPieceCtas && blk.tok_o == nullptr) {
         int k = st->sm_count / rem;
         if (k > 8) k = 8;
         if (k > n_tiles / 4) k = n_tiles / 4;
@@ -352,7 +356,12 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
                        qk_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
         if (rc != REGENVC_OK) return rc;
     }
-    CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, stream));
+    if (persistent) {
+        const int n_ctas = n_items < st->sm_count ? n_items : st->sm_count;
+        CUDA_TRY(launch_attn_persistent(tmap_k, tmap_v, tmap_out, tmap_q, ap, n_ctas, stream));
+    } else {
+        CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, stream));
+    }
     launched();
     if (ap.split_k > 1) {
         MergeParams mp;
@@ -815,7 +824,7 @@ int regenvc_device_status(void* stream, int* status_out) {
 }
 
 int regenvc_debug_set_phases(int mask) {
-    if (mask < 1 || mask > 3) return REGENVC_ERR_BAD_SHAPE;
+    if (mask < 1 || mask > 7 || !(mask & 3)) return REGENVC_ERR_BAD_SHAPE;
     tl_phases = mask;
     return REGENVC_OK;
 }

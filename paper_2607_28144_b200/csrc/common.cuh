@@ -135,6 +135,11 @@ cudaError_t launch_prep_kv(const PrepParams& p, cudaStream_t stream);
 // K'); nullptr: the kernel reads p.q (bf16), rotates if p.rope and converts to fp16 itself.
 cudaError_t launch_attn_pipelined(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
                                   const CUtensorMap* tmap_q, const AttnParams& p, cudaStream_t stream);
+// Persistent form for short key sequences (one CTA per SM walks over its work items; query tiles by TMA only).
+constexpr int kPersistentMaxTiles = 8;
+cudaError_t configure_attn_persistent();
+cudaError_t launch_attn_persistent(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
+                                   const CUtensorMap& tmap_q, const AttnParams& p, int n_ctas, cudaStream_t stream);
 cudaError_t configure_attn_pipelined();   // once per device: register hand-over check, large dynamic shared memory
 cudaError_t launch_merge_partials(const MergeParams& p, cudaStream_t stream);
 cudaError_t launch_merge_token_partials(const TokenMergeParams& p, cudaStream_t stream);
