@@ -357,7 +357,13 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
         if (rc != REGENVC_OK) return rc;
     }
     if (persistent) {
-        const int n_ctas = n_items < st->sm_count ? n_items : st->sm_count;
+        // a last round that would keep at most half of the SMs busy is handed out as single 128-row query tiles
+        int n_ctas = n_items < st->sm_count ? n_items : st->sm_count;
+        if (n_items > st->sm_count && rem > 0 && 2 * rem <= st->sm_count) ap.n_full_items = n_items - rem;
+        if (n_items <= st->sm_count / 2) {
+            ap.n_full_items = 0;
+            n_ctas = 2 * n_items;
+        }
         CUDA_TRY(launch_attn_persistent(tmap_k, tmap_v, tmap_out, tmap_q, ap, n_ctas, stream));
     } else {
         CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, stream));

@@ -9,9 +9,13 @@
 //     accumulator columns are handed back through o_free when the softmax warps have loaded them);
 //   * barriers, tensor memory and the tensor maps are set up once per CTA.
 // Roles, tensor-memory map, softmax scheme and the UMMA sequences are those of attn_pipelined.cu.  Shared memory:
-// Q0, Q1, a 3-slot K'/V't ring and one 32 KB staging tile for the output (the query buffers cannot double as
+// Q0, Q1, a 4-slot K'/V't ring and one 32 KB staging tile for the output (the query buffers cannot double as
 // staging here because the next item's tiles arrive while the epilogue runs; writing the output rows straight
 // from registers, 16 bytes per thread and store, was measured 13 us slower per call at the 480x832 window).
+// That is 7 tiles of 32 KB; with the barriers and one 2 KB row-exchange array it fits only because the dynamic
+// shared memory of a kernel without static shared memory starts on a 1024-byte boundary (checked at run time).
+// Work items: the first n_full_items are (head, 256 query rows); the items after them are single 128-row query
+// tiles, which the host uses for the last, incomplete round so that it is spread over twice as many SMs.
 // Only normalised bf16 output is produced (no key-range pieces, no token-major partial results).
 #include "attn_core.cuh"
 #include "common.cuh"
@@ -20,8 +24,29 @@ namespace regenvc {
 
 namespace {
 
-constexpr int kPStages = 3;
-constexpr uint32_t kPSmemBytes = (2 + kPStages + 1) * kTileBytes + 1024 /*align*/ + 256 /*barriers*/ + 8192 /*row exchange*/;
+constexpr int kPStages = 4;
+constexpr uint32_t kPXchBytes = kTile * kSplit * 4;   // one [128 rows][kSplit] float array for every row exchange
+constexpr uint32_t kPSmemBytes = (2 + kPStages + 1) * kTileBytes + 256 /*barriers*/ + kPXchBytes;
+static_assert(kPSmemBytes <= 232448, "shared memory of one SM");
+
+// A work item of the persistent kernel: head, first query row, number of 128-row query tiles (2, 1 or 0).
+struct PItem {
+    int head, q0, n_active;
+};
+__device__ __forceinline__ PItem decode_item(int item, const AttnParams& p) {
+    PItem w;
+    if (item < p.n_full_items) {
+        w.head = item / p.pairs_per_head;
+        w.q0 = (item % p.pairs_per_head) * 2 * kTile;
+        w.n_active = w.q0 + kTile < p.n_q ? 2 : 1;
+    } else {
+        const int hx = item - p.n_full_items, pair = p.n_full_items + (hx >> 1);
+        w.head = pair / p.pairs_per_head;
+        w.q0 = (pair % p.pairs_per_head) * 2 * kTile + (hx & 1) * kTile;
+        w.n_active = w.q0 < p.n_q ? 1 : 0;   // the second half of a pair whose second tile does not exist: no work
+    }
+    return w;
+}
 
 struct PBarriers {
     uint64_t kv_full[kPStages];
@@ -74,18 +99,25 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
                        const __grid_constant__ CUtensorMap tmap_out, const __grid_constant__ CUtensorMap tmap_q,
                        const AttnParams p) {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* base = smem_raw;
+    if ((smem_u32(base) & 1023u) != 0) {  // the swizzled tiles need a 1024-byte aligned base (uniform over the grid)
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusTimeout);
+        return;
+    }
     uint8_t* sQ = base;                                   // 2 tiles
     uint8_t* sKV = base + 2 * kTileBytes;                 // ring
     uint8_t* sOut = base + (2 + kPStages) * kTileBytes;   // staging tile of the epilogue
     PBarriers* bar = reinterpret_cast<PBarriers*>(base + (3 + kPStages) * kTileBytes);
-    RowExchange* xch = reinterpret_cast<RowExchange*>(base + (3 + kPStages) * kTileBytes + 256);
+    // values the kSplit threads of a row hand each other (tile maxima on the redo path, row sums in the epilogue;
+    // every use is fenced off from the next by a barrier of the threads involved, so one array serves all)
+    float (*xch)[kSplit] = reinterpret_cast<float (*)[kSplit]>(base + (3 + kPStages) * kTileBytes + 256);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     uint32_t tmem_base = 0;
     const WaitCtl ctl{&bar->abort_flag, p.status, kStatusTimeout, kWaitLimitNs};
     const int n_tiles = p.n_kv_pad / kTile;
-    const int n_items = p.pairs_per_head * p.h;
+    const int n_pairs = p.pairs_per_head * p.h;
+    const int n_items = p.n_full_items + 2 * (n_pairs - p.n_full_items);
     const int first_item = blockIdx.x, item_step = gridDim.x;
 
     if (warp >= kMmaWarp) {
@@ -128,10 +160,10 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
         if (elect_one()) {
             int kv_i = 0, it = 0;  // running ring index over all items, item count
             bool ok = true;
-            for (int item = first_item; ok && item < n_items; item += item_step, ++it) {
-                const int head = item / p.pairs_per_head;
-                const int q0 = (item % p.pairs_per_head) * 2 * kTile;
-                const int n_active = q0 + kTile < p.n_q ? 2 : 1;
+            for (int item = first_item; ok && item < n_items; item += item_step) {
+                const PItem w = decode_item(item, p);
+                const int head = w.head, q0 = w.q0, n_active = w.n_active;
+                if (n_active == 0) continue;  // every role skips an empty item the same way
                 for (int t = 0; ok && t < n_active; ++t) {
                     if (it > 0) ok = mbar_wait(smem_u32(&bar->q_empty[t]), (it - 1) & 1, ctl);
                     if (!ok) break;
@@ -157,6 +189,7 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
                         tma_load_2d(dst + kBlockBytes, &tmap_v, kv0 + 64, head * kHeadDim, full);
                     }
                 }
+                ++it;
             }
         }
       } else if (warp == kMmaWarp) {
@@ -167,9 +200,9 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
             int kv_c = 0, it = 0;       // ring index of the next tile to consume, item count
             int visit = 0;              // key tiles done so far over all items: the phase of s/p/o_full of BOTH tiles
             bool ok = true;
-            for (int item = first_item; ok && item < n_items; item += item_step, ++it) {
-                const int q0 = (item % p.pairs_per_head) * 2 * kTile;
-                const int n_active = q0 + kTile < p.n_q ? 2 : 1;
+            for (int item = first_item; ok && item < n_items; item += item_step) {
+                const int n_active = decode_item(item, p).n_active;
+                if (n_active == 0) continue;
                 for (int t = 0; ok && t < n_active; ++t) ok = mbar_wait(smem_u32(&bar->q_full[t]), it & 1, ctl);
                 if (ok) ok = mbar_wait(smem_u32(&bar->kv_full[kv_c % kPStages]), (kv_c / kPStages) & 1, ctl);
                 if (!ok) break;
@@ -223,6 +256,7 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
                     }
                     kv_c += more ? 2 : 1;
                 }
+                ++it;
             }
         }
       }
@@ -244,7 +278,8 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
         int visit = 0;  // key tiles done so far over all items = completed phases of s_full, p_full, o_full (both tiles)
 
         for (int item = first_item; item < n_items; item += item_step) {
-            const int n_active = (item % p.pairs_per_head) * 2 * kTile + kTile < p.n_q ? 2 : 1;
+            const int n_active = decode_item(item, p).n_active;
+            if (n_active == 0) continue;
             float m_ref[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
 
             for (int j = 0; j < n_tiles; ++j, ++visit) {
@@ -299,11 +334,11 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
                             mx3 = max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
                         }
                         const float mx_part = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                        xch->m[t][row][part] = mx_part;
+                        xch[row][part] = mx_part;
                         row_group_barrier(warp & 3);
                         float mx_row = mx_part;
 #pragma unroll
-                        for (int o = 1; o < kSplit; ++o) mx_row = fmaxf(mx_row, xch->m[t][row][(part + o) % kSplit]);
+                        for (int o = 1; o < kSplit; ++o) mx_row = fmaxf(mx_row, xch[row][(part + o) % kSplit]);
                         row_group_barrier(warp & 3);
                         const float m_tile = mx_row * scale;
                         const bool raise = m_tile > m_ref[t];
@@ -351,52 +386,55 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
 #pragma unroll 1
             for (int t = 0; t < 2; ++t) {
                 if (t < n_active) {
-                    xch->l[t][row][part] = l_run[t];
-                    // the staging tile is free once the previous store has read it (thread 0 issued it)
-                    if (tid == 0) tma_store_wait_read();
+                    xch[row][part] = l_run[t];
                     softmax_barrier();
                     float l_row = 0.f;
 #pragma unroll
-                    for (int o = 0; o < kSplit; ++o) l_row += xch->l[t][row][o];
+                    for (int o = 0; o < kSplit; ++o) l_row += xch[row][o];
                     const float inv_l = 1.0f / l_row;
                     if (ok) ok = mbar_wait_lean(bars, kOffOFull + 8 * t, (visit - 1) & 1, p.status);
                     ok = __all_sync(0xffffffffu, ok);
                     tc_fence_after();
-                    const uint32_t t_O = t_S0 + 256 + t * 128;
-#pragma unroll 1
-                    for (int cb = 0; cb < kChunks; ++cb) {
+                    static_assert(kChunks == 1, "the epilogue keeps one 32-column chunk per thread in registers");
+                    uint4 w[4];
+                    if (ok) {
                         uint32_t o[32];
-                        if (ok) {
-                            tmem_ld32(t_O + cb * 32, o);
-                            tmem_wait_ld();
+                        tmem_ld32(t_S0 + 256 + t * 128, o);
+                        tmem_wait_ld();
 #pragma unroll
-                            for (int c = 0; c < 4; ++c) {
-                                uint4 w;
-                                w.x = pack_bf16x2(__uint_as_float(o[8 * c + 0]) * inv_l, __uint_as_float(o[8 * c + 1]) * inv_l);
-                                w.y = pack_bf16x2(__uint_as_float(o[8 * c + 2]) * inv_l, __uint_as_float(o[8 * c + 3]) * inv_l);
-                                w.z = pack_bf16x2(__uint_as_float(o[8 * c + 4]) * inv_l, __uint_as_float(o[8 * c + 5]) * inv_l);
-                                w.w = pack_bf16x2(__uint_as_float(o[8 * c + 6]) * inv_l, __uint_as_float(o[8 * c + 7]) * inv_l);
-                                const int col = part * kColsPerThread + cb * 32 + c * 8;
-                                *reinterpret_cast<uint4*>(sOut + (col >> 6) * kBlockBytes + sw128_offset(row, (col >> 3) & 7)) = w;
-                            }
+                        for (int c = 0; c < 4; ++c) {
+                            w[c].x = pack_bf16x2(__uint_as_float(o[8 * c + 0]) * inv_l, __uint_as_float(o[8 * c + 1]) * inv_l);
+                            w[c].y = pack_bf16x2(__uint_as_float(o[8 * c + 2]) * inv_l, __uint_as_float(o[8 * c + 3]) * inv_l);
+                            w[c].z = pack_bf16x2(__uint_as_float(o[8 * c + 4]) * inv_l, __uint_as_float(o[8 * c + 5]) * inv_l);
+                            w[c].w = pack_bf16x2(__uint_as_float(o[8 * c + 6]) * inv_l, __uint_as_float(o[8 * c + 7]) * inv_l);
                         }
                     }
-                }
-                // the accumulator columns of this tile may be overwritten by the next item (arrives once per item and
-                // tile, also for a tile that does not exist, so that the barrier's phase follows the item count)
-                tc_fence_before();
-                mbar_arrive_at(bars, kOffOFree + 8 * t);
-                if (t < n_active) {
+                    // the accumulator columns of this tile may now be overwritten by the next item
+                    tc_fence_before();
+                    mbar_arrive_at(bars, kOffOFree + 8 * t);
+                    // the staging tile is free once the previous store has read it (thread 0 issued that store); by now
+                    // that read has had the time of the row-sum exchange and of the accumulator load to finish
+                    if (tid == 0) tma_store_wait_read();
+                    softmax_barrier();
+                    if (ok) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const int col = part * kColsPerThread + c * 8;
+                            *reinterpret_cast<uint4*>(sOut + (col >> 6) * kBlockBytes + sw128_offset(row, (col >> 3) & 7)) = w[c];
+                        }
+                    }
                     fence_proxy_async_smem();
                     softmax_barrier();
                     if (tid == 0 && ok) {
-                        const int head = item / p.pairs_per_head;
-                        const int q0 = (item % p.pairs_per_head) * 2 * kTile;
+                        const PItem wi = decode_item(item, p);
                         const uint32_t src = smem_u32(sOut);
-                        tma_store_2d(&tmap_out, head * kHeadDim, q0 + t * kTile, src);
-                        tma_store_2d(&tmap_out, head * kHeadDim + 64, q0 + t * kTile, src + kBlockBytes);
+                        tma_store_2d(&tmap_out, wi.head * kHeadDim, wi.q0 + t * kTile, src);
+                        tma_store_2d(&tmap_out, wi.head * kHeadDim + 64, wi.q0 + t * kTile, src + kBlockBytes);
                         tma_store_commit();
                     }
+                } else {
+                    // a tile that does not exist still arrives, so that the barrier's phase follows the item count
+                    mbar_arrive_at(bars, kOffOFree + 8 * t);
                 }
             }
         }
