@@ -6,7 +6,10 @@
 
 One "step" is one pass of the whole hot path over one window: the
 self-attention call (key/value preparation pass + attention kernel) followed by
-one cross-attention call per conditioning sequence of the workload.  At N = 1
+one cross-attention call per conditioning sequence of the workload, on
+conditioning operands that were prepared once before the timed region (the
+paper computes the conditioning keys/values once per sequence, Sec. 3.9; the
+step with that preparation inside every call is timed as well).  At N = 1
 the workload is the 480x832 window (7x30x52 = 10920 tokens, 12 heads x 128,
 plus 512 conditioning tokens), the shape the tensor-peak target is quoted on.
 With N > 1 (one process per GPU under torchrun; without a launcher the script
@@ -297,6 +300,9 @@ def run_ours(args, w: synth.Workload):
         sets.append({"q": q.to(dev), "k": k.to(dev), "v": v.to(dev),
                      "cross": [(a.to(dev), b.to(dev)) for a, b in cross],
                      "out": torch.empty_like(q, device=dev), "outc": [torch.empty_like(q, device=dev) for _ in cross],
+                     # the conditioning keys/values are computed once per sequence (Sec. 3.9): their operand form is
+                     # prepared here, once, and every timed step runs the cross-attention call on it
+                     "prepared": [binding.regenvc_cross_kv_prepare(a.to(dev), b.to(dev)) for a, b in cross],
                      # a workspace of its own, used only where the attention kernel is timed alone: the operands
                      # prepared from this set's k and v stay in it between launches
                      "ws": torch.empty((binding.regenvc_workspace_bytes(w.n_tokens, w.n_heads),), dtype=torch.uint8,
@@ -305,6 +311,11 @@ def run_ours(args, w: synth.Workload):
     stream = torch.cuda.Stream(device=dev)
 
     def step(s):
+        binding.regenvc_attn_forward(s["q"], s["k"], s["v"], s["out"], w.T, w.H, w.W, w.theta, stream)
+        for prep, n_kv, oc in zip(s["prepared"], w.cross_kv, s["outc"]):
+            binding.regenvc_cross_attn_forward_prepared(s["q"], prep, n_kv, oc, stream)
+
+    def step_one_call_cross(s):
         binding.regenvc_attn_forward(s["q"], s["k"], s["v"], s["out"], w.T, w.H, w.W, w.theta, stream)
         for (ck, cv), oc in zip(s["cross"], s["outc"]):
             binding.regenvc_cross_attn_forward(s["q"], ck, cv, oc, stream)
@@ -366,6 +377,15 @@ def run_ours(args, w: synth.Workload):
         status = binding.regenvc_device_status(stream)
         if status != 0:
             raise SystemExit(f"device status {status}: {binding.status_string(status)}")
+
+        # the same steps with the conditioning operands rewritten inside every cross-attention call, for comparison
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(stream)
+        for i in range(args.steps):
+            step_one_call_cross(sets[i % N_BUFFER_SETS])
+        g1.record(stream)
+        torch.cuda.synchronize()
+        ms_step_one_call = g0.elapsed_time(g1) / args.steps
 
         # ---- the dominant kernel alone, burst regime: isolated launches right after a pause
         time.sleep(0.5)
@@ -488,10 +508,13 @@ def run_ours(args, w: synth.Workload):
             "config": {"workload": w.name, "grid_THW": [w.T, w.H, w.W], "tokens": w.n_tokens, "heads": w.n_heads,
                        "head_dim": w.head_dim, "cross_kv": list(w.cross_kv), "layers": w.layers,
                        "denoise_steps": w.steps, "parallelism": f"{world} independent window(s), one per GPU",
+                       "cross_attention": "on conditioning operands prepared once per sequence "
+                                          "(regenvc_cross_kv_prepare, outside the timed steps)",
                        "communicator_ranks": ranks_seen,
                        "l2": f"{N_BUFFER_SETS} rotating input sets, each {4 * w.n_tokens * w.n_heads * 256 / 1e6:.0f} MB "
                              f"of q/k/v/out (L2 is 126 MB)"},
             "ms_per_window": ms_step * w.layers * w.steps,
+            "ms_per_step_cross_prepared_in_call": ms_step_one_call,
             "pct_of_nominal_2250": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
             "gpu_launches": int(launches),
             "clocks": sampler.summary(),
