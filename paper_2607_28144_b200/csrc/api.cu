@@ -627,7 +627,7 @@ int regenvc_qkv_rope_project(const void* x, const void* w_qkv, const void* b_qkv
     if (rc == REGENVC_OK)
         rc = make_tmap(&tmap_v, vt, (uint64_t)n_pad, (uint64_t)n_heads * kHeadDim, (uint64_t)n_pad * sizeof(__half));
     if (rc != REGENVC_OK) return rc;
-    CUDA_TRY(launch_qkv_project(tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, pp, (cudaStream_t)stream));
+    CUDA_TRY(launch_qkv_project(tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, pp, st->sm_count, (cudaStream_t)stream));
     launched();
     return REGENVC_OK;
 }

@@ -68,7 +68,7 @@ struct AttnParams {
 };
 
 // QKV projection with fused norm / rotation / operand-layout epilogue (producer of the attention operands).
-constexpr int kProjHeadsPerCta = 2;   // a CTA computes 128 tokens x two heads of one of q, k, v
+constexpr int kProjHeadsPerCta = 2;   // a CTA computes 128 tokens x two heads of one of q, k, v per work unit
 constexpr int kProjMaxCluster = 8;    // the CTAs that share a token tile form one cluster (h / 2 of them)
 struct ProjParams {
     const float* bias;        // [3C] or nullptr
@@ -82,7 +82,7 @@ struct ProjParams {
 cudaError_t configure_qkv_project();
 cudaError_t launch_qkv_project(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w, const CUtensorMap& tmap_q,
                                const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const ProjParams& p,
-                               cudaStream_t stream);
+                               int sm_count, cudaStream_t stream);
 
 // Merge of token-major partial results of several key/value blocks.
 constexpr int kMaxMergeParts = 8;

@@ -7,16 +7,20 @@
 //   V't fp16 [h][128][n_pad]      values, keys contiguous       } so no separate preparation pass is needed
 // and nothing of q, k, v is ever rounded to bf16 or written in token-major form.
 //
-// One CTA computes 128 tokens x 256 output features (two heads) of one of q, k, v:
-//   warp 0      TMA producer: x tile [128 tokens][64] and W tile [256 features][64] per stage (bf16, 128B swizzle)
-//   warp 1      tcgen05.mma issuer (bf16 x bf16 -> fp32 in 256 tensor-memory columns) and TMEM owner
+// A work unit is (128-token tile, one of q / k / v); the h/2 CTAs of a thread-block cluster compute it together,
+// each 256 output features (two heads).  Clusters are persistent: cluster c takes units c, c + n_clusters, ...
+//   warp 0      TMA producer: x tile [128 tokens][64] and W tile [256 features][64] per stage (bf16, 128B swizzle),
+//               a 3-stage ring that runs on into the next unit
+//   warp 1      tcgen05.mma issuer (bf16 x bf16 -> fp32) and TMEM owner; two accumulators of 256 columns, used in
+//               turn, so that the main loop of one unit runs while the epilogue warps empty the other accumulator
 //   warps 2-9   epilogue, two threads per accumulator row (one per head)
 // q and k: D[token][feature] = x W^T (A = x tile, B = W tile, N = 256).  v: D[feature][token] = W x^T (A = W rows of
 // one head, B = x tile), which is V't directly -- no transpose anywhere.
-// The RMS norm needs the sum of squares over ALL features of a token, which are spread over the h/2 CTAs that
-// share the token tile: those CTAs form a thread-block cluster and read each other's partial row sums through
-// distributed shared memory.  96 KB of shared memory and 256 tensor-memory columns per CTA: two CTAs share an SM,
-// so one's epilogue overlaps the other's main loop.
+// The RMS norm needs the sum of squares over ALL features of a token, which are spread over the CTAs of the cluster:
+// every CTA writes its partial row sums into the shared memory of all of them (distributed shared memory) and
+// arrives on their barriers; only the epilogue warps wait for it, the producer and the MMA warp run ahead.
+#include <cstddef>
+
 #include "common.cuh"
 #include "ptx.cuh"
 #include "rope.cuh"
@@ -27,7 +31,7 @@ namespace regenvc {
 namespace {
 
 constexpr int kBK = 64;                                  // K elements per stage: one 128-byte swizzled row
-constexpr int kProjStages = 2;
+constexpr int kProjStages = 3;
 constexpr int kFeat = kProjHeadsPerCta * kHeadDim;       // 256 output features per CTA
 constexpr uint32_t kXBytes = kTile * kBK * 2;            // 16 KB
 constexpr uint32_t kWBytes = kFeat * kBK * 2;            // 32 KB
@@ -36,21 +40,26 @@ constexpr int kEpiThreads = 256;
 constexpr int kProjThreads = 64 + kEpiThreads;
 constexpr uint32_t kOutTileBytes = kTile * kHeadDim * 2; // 32 KB: one head's [128][128] fp16 tile, staged for TMA
 constexpr uint32_t kOutBlockBytes = kOutTileBytes / 2;
-static_assert(kProjHeadsPerCta * kOutTileBytes <= kProjStages * kStageBytes, "output staging reuses the stage buffers");
-constexpr uint32_t kProjSmem = kProjStages * kStageBytes + 1024 /*align*/ + 128 /*barriers*/ +
-                               2 * kFeat * 4 /*bias, gain*/ + 3 * kTile * 4 /*row sums*/;
 constexpr uint64_t kProjWaitNs = 500000000ull;
 constexpr uint32_t kIdescQK = umma_idesc_bf16_f32acc(128, kFeat);
 constexpr uint32_t kIdescV = umma_idesc_bf16_f32acc(128, 128);
 
-struct ProjBarriers {
+struct ProjShared {
     uint64_t full[kProjStages];
     uint64_t empty[kProjStages];
-    uint64_t acc_full;
+    uint64_t acc_full[2];      // accumulator b holds a finished unit
+    uint64_t acc_empty[2];     // the epilogue has read accumulator b out
+    uint64_t sums_in[2];       // every CTA of the cluster has delivered its partial row sums into xsum[b]
     uint32_t tmem_base;
     int abort_flag;
+    float bias[kFeat];         // this unit's slice of the bias
+    float gain[kFeat];         //             ... and of the norm gains
+    float part[2][kTile];      // partial sums of squares of the two heads of this CTA
+    float xsum[2][kProjMaxCluster][kTile];  // [buffer][source CTA][token]: partial row sums of the whole cluster
 };
-static_assert(sizeof(ProjBarriers) <= 128, "barrier block too large");
+constexpr uint32_t kProjSmem = kProjStages * kStageBytes + kProjHeadsPerCta * kOutTileBytes + 1024 /*align*/ +
+                               sizeof(ProjShared);
+static_assert(kProjSmem <= 232448, "shared memory of one SM");
 
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 __device__ __forceinline__ void cluster_sync_all() {
@@ -61,242 +70,350 @@ __device__ __forceinline__ uint32_t cluster_size() {
     asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(n));
     return n;
 }
-// Reads a float at the same shared-memory offset in CTA `rank` of this cluster.
-__device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t rank) {
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t n;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(n));
+    return n;
+}
+__device__ __forceinline__ uint32_t cluster_id_x() {
+    uint32_t n;
+    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(n));
+    return n;
+}
+__device__ __forceinline__ uint32_t n_clusters_x() {
+    uint32_t n;
+    asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(n));
+    return n;
+}
+// Address of the same shared-memory location in CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
     uint32_t remote;
-    float v;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
-    return v;
+    return remote;
+}
+// Asynchronous 4-byte store into the shared memory of a CTA of the cluster that counts its bytes on a barrier of that
+// same CTA: whoever sees the barrier's phase complete (acquire at cluster scope) sees the value.  No fence is needed
+// on the sending side (a release-arrive per store, tried first, cost about 1.7 k clocks each).
+__device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float v, uint32_t cluster_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                 ::"r"(cluster_addr), "r"(__float_as_uint(v)), "r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, const WaitCtl& ctl) {
+    uint64_t t0 = 0;
+    uint32_t spins = 0;
+    while (!mbar_try_wait_cluster(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*ctl.abort_flag) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > ctl.limit_ns) {
+                *ctl.abort_flag = 1;
+                atomicCAS(ctl.status, 0, ctl.code);
+                return false;
+            }
+        }
+    }
+    return true;
 }
 
 }  // namespace
 
-__global__ void __launch_bounds__(kProjThreads, 2)
+__global__ void __launch_bounds__(kProjThreads, 1)
 qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                    const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                    const __grid_constant__ CUtensorMap tmap_v, const ProjParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* stages = base;
-    ProjBarriers* bar = reinterpret_cast<ProjBarriers*>(base + kProjStages * kStageBytes);
-    float* bias_s = reinterpret_cast<float*>(base + kProjStages * kStageBytes + 128);
-    float* gain_s = bias_s + kFeat;
-    float* part_s = gain_s + kFeat;          // [2][128] partial sums of squares of the two column halves
-    float* rowsum_s = part_s + 2 * kTile;    // [128]    this CTA's sum of squares per token, read by the cluster
+    uint8_t* stage_out = base + kProjStages * kStageBytes;   // two [128][128] fp16 tiles for the tiled stores
+    ProjShared* sh = reinterpret_cast<ProjShared*>(stage_out + kProjHeadsPerCta * kOutTileBytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int pair = blockIdx.x;             // which two heads (= rank in the cluster)
-    const int n0 = blockIdx.y * kTile;       // first token of the tile
-    const int part = blockIdx.z;             // 0 q, 1 k, 2 v
-    const int f0 = part * p.C + pair * kFeat;  // first row of W_qkv (output feature) of this CTA
+    const int pair = static_cast<int>(cluster_rank());       // which two heads
+    const int n_rank = static_cast<int>(cluster_size());
+    const int n_tiles = (p.n_tokens + kTile - 1) / kTile;
+    const int n_units = 3 * n_tiles;                         // unit u: token tile u / 3, part u % 3 (0 q, 1 k, 2 v)
+    const int unit0 = static_cast<int>(cluster_id_x()), unit_step = static_cast<int>(n_clusters_x());
     const int n_kb = p.C / kBK;
-    const WaitCtl ctl{&bar->abort_flag, p.status, kStatusTimeout, kProjWaitNs};
+    const WaitCtl ctl{&sh->abort_flag, p.status, kStatusTimeout, kProjWaitNs};
     uint32_t tmem_base = 0;
 
     if (tid == 0) {
         for (int s = 0; s < kProjStages; ++s) {
-            mbar_init(smem_u32(&bar->full[s]), 1);
-            mbar_init(smem_u32(&bar->empty[s]), 1);
+            mbar_init(smem_u32(&sh->full[s]), 1);
+            mbar_init(smem_u32(&sh->empty[s]), 1);
         }
-        mbar_init(smem_u32(&bar->acc_full), 1);
-        bar->abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0) ? 1 : 0;
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&sh->acc_full[b]), 1);
+            mbar_init(smem_u32(&sh->acc_empty[b]), kEpiThreads);
+            mbar_init(smem_u32(&sh->sums_in[b]), 1);   // one local arrival that announces the bytes, then the bytes
+        }
+        sh->abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0) ? 1 : 0;
         fence_mbar_init();
     }
     __syncwarp();
     if (warp == 1) {
-        tmem_alloc(smem_u32(&bar->tmem_base), kFeat);
+        tmem_alloc(smem_u32(&sh->tmem_base), 512);
         tmem_relinquish();
-    }
-    if (warp >= 2) {
-        // this CTA's slice of the bias and of the norm gains, once
-        const int t = tid - 64;
-        bias_s[t] = p.bias ? __ldg(p.bias + f0 + t) : 0.0f;
-        const float* g = part == 0 ? p.g_q : p.g_k;
-        gain_s[t] = (part < 2 && g) ? __ldg(g + pair * kFeat + t) : 1.0f;
     }
     tc_fence_before();
     __syncthreads();
+    // nobody may arrive on a barrier of another CTA before that CTA has initialised it
+    cluster_sync_all();
     tc_fence_after();
-    tmem_base = bar->tmem_base;
+    tmem_base = sh->tmem_base;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
             tma_prefetch_desc(&tmap_x);
             tma_prefetch_desc(&tmap_w);
-            for (int kb = 0; kb < n_kb; ++kb) {
-                const int s = kb % kProjStages, round = kb / kProjStages;
-                if (round > 0 && !mbar_wait(smem_u32(&bar->empty[s]), (round - 1) & 1, ctl)) break;
-                const uint32_t full = smem_u32(&bar->full[s]);
-                const uint32_t dst = smem_u32(stages + s * kStageBytes);
-                mbar_expect_tx(full, kStageBytes);
-                tma_load_2d(dst, &tmap_x, kb * kBK, n0, full);             // rows past the last token arrive as zeros
-                tma_load_2d(dst + kXBytes, &tmap_w, kb * kBK, f0, full);
+            int fill = 0;  // stages filled so far over all units
+            bool ok = true;
+            for (int unit = unit0; ok && unit < n_units; unit += unit_step) {
+                const int n0 = (unit / 3) * kTile;
+                const int f0 = (unit % 3) * p.C + pair * kFeat;   // first row of W_qkv (output feature) of this CTA
+                for (int kb = 0; kb < n_kb; ++kb, ++fill) {
+                    const int s = fill % kProjStages, round = fill / kProjStages;
+                    if (round > 0) ok = mbar_wait(smem_u32(&sh->empty[s]), (round - 1) & 1, ctl);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&sh->full[s]);
+                    const uint32_t dst = smem_u32(stages + s * kStageBytes);
+                    mbar_expect_tx(full, kStageBytes);
+                    tma_load_2d(dst, &tmap_x, kb * kBK, n0, full);   // rows past the last token arrive as zeros
+                    tma_load_2d(dst + kXBytes, &tmap_w, kb * kBK, f0, full);
+                }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (elect_one()) {
+            int fill = 0, it = 0;
             bool ok = true;
-            for (int kb = 0; kb < n_kb && ok; ++kb) {
-                const int s = kb % kProjStages;
-                ok = mbar_wait(smem_u32(&bar->full[s]), (kb / kProjStages) & 1, ctl);
+            for (int unit = unit0; ok && unit < n_units; unit += unit_step, ++it) {
+                const int part = unit % 3, b = it & 1;
+                const uint32_t acc_tmem = tmem_base + b * kFeat;
+                // the accumulator must have been read out by the epilogue of the unit before last
+                if (it >= 2) ok = mbar_wait(smem_u32(&sh->acc_empty[b]), ((it >> 1) - 1) & 1, ctl);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t sx = smem_u32(stages + s * kStageBytes), sw = sx + kXBytes;
-                const uint64_t dx = umma_smem_desc_k_sw128(sx), dw = umma_smem_desc_k_sw128(sw);
+                for (int kb = 0; kb < n_kb; ++kb, ++fill) {
+                    const int s = fill % kProjStages;
+                    ok = mbar_wait(smem_u32(&sh->full[s]), (fill / kProjStages) & 1, ctl);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sx = smem_u32(stages + s * kStageBytes), sw = sx + kXBytes;
+                    const uint64_t dx = umma_smem_desc_k_sw128(sx), dw = umma_smem_desc_k_sw128(sw);
 #pragma unroll
-                for (int kk = 0; kk < kBK / 16; ++kk) {
-                    const uint32_t acc = (kb > 0 || kk > 0) ? 1u : 0u;
-                    if (part < 2) {
-                        umma_ss(tmem_base, dx + 2 * kk, dw + 2 * kk, kIdescQK, acc);
-                    } else {
+                    for (int kk = 0; kk < kBK / 16; ++kk) {
+                        const uint32_t acc = (kb > 0 || kk > 0) ? 1u : 0u;
+                        if (part < 2) {
+                            umma_ss(acc_tmem, dx + 2 * kk, dw + 2 * kk, kIdescQK, acc);
+                        } else {
 #pragma unroll
-                        for (int i = 0; i < kProjHeadsPerCta; ++i)
-                            umma_ss(tmem_base + i * 128, dw + i * ((kTile * kBK * 2) >> 4) + 2 * kk, dx + 2 * kk, kIdescV, acc);
+                            for (int i = 0; i < kProjHeadsPerCta; ++i)
+                                umma_ss(acc_tmem + i * 128, dw + i * ((kTile * kBK * 2) >> 4) + 2 * kk, dx + 2 * kk,
+                                        kIdescV, acc);
+                        }
+                    }
+                    umma_commit(smem_u32(&sh->empty[s]));
+                }
+                if (ok) umma_commit(smem_u32(&sh->acc_full[b]));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        const int half = (warp - 2) >> 2;             // which head of the CTA's two this thread works on
+        const int row = (warp & 3) * 32 + lane;       // accumulator row = TMEM lane
+        const int et = tid - 64;                      // 0 .. 255
+        uint8_t* my_stage = stage_out + half * kOutTileBytes;
+        bool ok = true;
+        int it = 0, normed_seen = 0;
+        for (int unit = unit0; unit < n_units; unit += unit_step, ++it) {
+            const int part = unit % 3, n0 = (unit / 3) * kTile, b = it & 1;
+            const bool normed = part < 2;
+            const uint32_t t_acc = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + b * kFeat + half * 128;
+            // this unit's slice of the bias and of the norm gains (the previous unit's readers are past the barrier
+            // that closed its epilogue)
+            {
+                const int f0 = part * p.C + pair * kFeat;
+                sh->bias[et] = p.bias ? __ldg(p.bias + f0 + et) : 0.0f;
+                const float* g = part == 0 ? p.g_q : p.g_k;
+                sh->gain[et] = (normed && g) ? __ldg(g + pair * kFeat + et) : 1.0f;
+            }
+            epi_barrier();
+            if (ok) ok = mbar_wait(smem_u32(&sh->acc_full[b]), (it >> 1) & 1, ctl);
+            ok = __all_sync(0xffffffffu, ok);
+            tc_fence_after();
+
+            float inv_rms = 1.0f;
+            if (normed) {
+                // pass 1: this thread's share of the sum of squares of its token's features
+                float ss = 0.f;
+                if (ok) {
+#pragma unroll 1
+                    for (int cb = 0; cb < 4; ++cb) {
+                        uint32_t a[32];
+                        tmem_ld32(t_acc + cb * 32, a);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            const float y = __uint_as_float(a[c]) + sh->bias[half * 128 + cb * 32 + c];
+                            ss = fmaf(y, y, ss);
+                        }
                     }
                 }
-                umma_commit(smem_u32(&bar->empty[s]));
+                sh->part[half][row] = ss;
+                epi_barrier();
+                const int xb = normed_seen & 1;
+                if (et == 0) mbar_expect_tx(smem_u32(&sh->sums_in[xb]), n_rank * kTile * 4);  // what this CTA will receive
+                if (half == 0) {
+                    // deliver this CTA's partial sum of the token to every CTA of the cluster (itself included)
+                    const float mine = sh->part[0][row] + sh->part[1][row];
+                    const uint32_t slot = smem_u32(&sh->xsum[xb][pair][row]), barx = smem_u32(&sh->sums_in[xb]);
+                    for (int r = 0; r < n_rank; ++r) st_async_f32(map_to_rank(slot, r), mine, map_to_rank(barx, r));
+                }
+                if (ok) ok = mbar_wait_cluster(smem_u32(&sh->sums_in[xb]), (normed_seen >> 1) & 1, ctl);
+                ok = __all_sync(0xffffffffu, ok);
+                float total = 0.f;
+                for (int r = 0; r < n_rank; ++r) total += sh->xsum[xb][r][row];
+                inv_rms = rsqrtf(total / static_cast<float>(p.C) + p.eps);
+                ++normed_seen;
             }
-            if (ok) umma_commit(smem_u32(&bar->acc_full));
-        }
-    }
-    __syncwarp();
 
-    const bool normed = part < 2;                      // uniform over the cluster
-    const int half = warp >= 2 ? (warp - 2) >> 2 : 0;  // which head of the CTA's two this thread works on
-    const int row = (warp & 3) * 32 + lane;            // accumulator row = TMEM lane
-    const uint32_t t_acc = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + half * 128;
-    bool ok = true;
-    float inv_rms = 1.0f;
-    if (warp >= 2) {
-        ok = mbar_wait(smem_u32(&bar->acc_full), 0, ctl);
-        ok = __all_sync(0xffffffffu, ok);
-        tc_fence_after();
-        if (normed) {
-            // pass 1: this thread's share of the sum of squares of its token's features
-            float ss = 0.f;
-            if (ok) {
+            // the staging tiles are free once the previous unit's stores have read them (thread 64 issued them)
+            if (tid == 64) tma_store_wait_read();
+            epi_barrier();
+            if (normed) {
+                const int n = n0 + row;
+                const bool live = n < p.n_tokens;
+                const TokenPos pos = token_pos(live ? n : 0, p.grid);
+                float amax = 0.f;  // largest magnitude of this row, for the fp16 range check
+                // Fully unrolled so that the place of every pair in the rotary table is a compile-time constant.  The 16
+                // (cos, sin) entries of a 32-column chunk are requested one chunk ahead, so that their latency (with
+                // two warps per scheduler nothing else hides it) falls on the arithmetic of the chunk before.
+                float2 cs_next[16];
+                auto fetch_cs = [&](int cbn, float2* dst) {
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        const RopeChunk rc = rope_chunk(p.grid, cbn * 4 + c8);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int at = rc.axis[i] == 0 ? pos.t : (rc.axis[i] == 1 ? pos.y : pos.x);
+                            dst[c8 * 4 + i] = __ldg(p.grid.tab + at * rc.mult[i] + rc.off[i]);
+                        }
+                    }
+                };
+                fetch_cs(0, cs_next);
+#pragma unroll
+                for (int cb = 0; cb < 4; ++cb) {
+                    float2 cs[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) cs[i] = cs_next[i];
+                    if (cb + 1 < 4) fetch_cs(cb + 1, cs_next);
+                    uint32_t a[32];
+                    if (ok) {
+                        tmem_ld32(t_acc + cb * 32, a);
+                        tmem_wait_ld();
+                    }
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        float x[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int col = half * 128 + cb * 32 + c8 * 8 + i;
+                            x[i] = (__uint_as_float(a[c8 * 8 + i]) + sh->bias[col]) * inv_rms * sh->gain[col];
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {  // pair (2i, 2i + 1) of this 8-column piece turns by its angle
+                            const float2 w2 = cs[c8 * 4 + i];
+                            const float xa = x[2 * i], xb2 = x[2 * i + 1];
+                            x[2 * i] = xa * w2.x - xb2 * w2.y;
+                            x[2 * i + 1] = xa * w2.y + xb2 * w2.x;
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            amax = fmaxf(amax, fabsf(x[i]));
+                            if (!live || !ok) x[i] = 0.f;   // padding rows of K' are zero
+                        }
+                        uint4 w;
+                        w.x = pack_f16x2(x[0], x[1]);
+                        w.y = pack_f16x2(x[2], x[3]);
+                        w.z = pack_f16x2(x[4], x[5]);
+                        w.w = pack_f16x2(x[6], x[7]);
+                        const int col = cb * 32 + c8 * 8;
+                        *reinterpret_cast<uint4*>(my_stage + (col >> 6) * kOutBlockBytes + sw128_offset(row, (col >> 3) & 7)) = w;
+                    }
+                }
+                if (!(amax <= 65504.0f) && live && ok) atomicCAS(p.status, 0, kStatusRange);
+            } else {
+                // v: row = feature of head `half`, columns = the tile's tokens
+                const float bv = sh->bias[half * 128 + row];
+                float vmax = 0.f;
 #pragma unroll 1
                 for (int cb = 0; cb < 4; ++cb) {
                     uint32_t a[32];
-                    tmem_ld32(t_acc + cb * 32, a);
-                    tmem_wait_ld();
+                    if (ok) {
+                        tmem_ld32(t_acc + cb * 32, a);
+                        tmem_wait_ld();
+                    }
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float y = __uint_as_float(a[c]) + bias_s[half * 128 + cb * 32 + c];
-                        ss = fmaf(y, y, ss);
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        float x[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int n = n0 + cb * 32 + c8 * 8 + i;
+                            x[i] = (ok && n < p.n_tokens) ? __uint_as_float(a[c8 * 8 + i]) + bv : 0.f;  // padding columns zero
+                            vmax = fmaxf(vmax, fabsf(x[i]));
+                        }
+                        uint4 w;
+                        w.x = pack_f16x2(x[0], x[1]);
+                        w.y = pack_f16x2(x[2], x[3]);
+                        w.z = pack_f16x2(x[4], x[5]);
+                        w.w = pack_f16x2(x[6], x[7]);
+                        const int col = cb * 32 + c8 * 8;
+                        *reinterpret_cast<uint4*>(my_stage + (col >> 6) * kOutBlockBytes + sw128_offset(row, (col >> 3) & 7)) = w;
                     }
                 }
+                if (!(vmax <= 65504.0f)) atomicCAS(p.status, 0, kStatusRange);
             }
-            part_s[half * kTile + row] = ss;
+            // the accumulator may be overwritten by the unit after next
+            tc_fence_before();
+            mbar_arrive(smem_u32(&sh->acc_empty[b]));
+            fence_proxy_async_smem();
             epi_barrier();
-            if (half == 0) rowsum_s[row] = part_s[row] + part_s[kTile + row];
-        }
-    }
-    if (normed) {
-        // every thread of every CTA of the cluster meets here: the partial sums are visible cluster-wide afterwards
-        __syncwarp();
-        cluster_sync_all();
-        if (warp >= 2) {
-            float total = 0.f;
-            const uint32_t n_rank = cluster_size();
-            for (uint32_t r = 0; r < n_rank; ++r) total += ld_cluster_f32(smem_u32(rowsum_s + row), r);
-            inv_rms = rsqrtf(total / static_cast<float>(p.C) + p.eps);
-        }
-    }
-
-    if (warp >= 2) {
-        bool out_of_range = false;
-        uint8_t* stage_out = stages + half * kOutTileBytes;  // the stage buffers are idle: all MMAs have completed
-        if (normed) {
-            const int n = n0 + row;
-            const bool live = n < p.n_tokens;
-            const TokenPos pos = token_pos(live ? n : 0, p.grid);
-#pragma unroll 1
-            for (int cb = 0; cb < 4; ++cb) {
-                uint32_t a[32];
-                if (ok) {
-                    tmem_ld32(t_acc + cb * 32, a);
-                    tmem_wait_ld();
-                }
+            if (tid == 64 && ok) {
 #pragma unroll
-                for (int c8 = 0; c8 < 4; ++c8) {
-                    float x[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int col = half * 128 + cb * 32 + c8 * 8 + i;
-                        x[i] = (__uint_as_float(a[c8 * 8 + i]) + bias_s[col]) * inv_rms * gain_s[col];
+                for (int i = 0; i < kProjHeadsPerCta; ++i) {
+                    const int head = pair * kProjHeadsPerCta + i;
+                    const uint32_t src = smem_u32(stage_out + i * kOutTileBytes);
+                    if (part == 0) {
+                        tma_store_2d(&tmap_q, head * kHeadDim, n0, src);
+                        tma_store_2d(&tmap_q, head * kHeadDim + 64, n0, src + kOutBlockBytes);
+                    } else if (part == 1) {
+                        tma_store_2d(&tmap_k, 0, head * p.n_pad + n0, src);
+                        tma_store_2d(&tmap_k, 64, head * p.n_pad + n0, src + kOutBlockBytes);
+                    } else {
+                        tma_store_2d(&tmap_v, n0, head * kHeadDim, src);
+                        tma_store_2d(&tmap_v, n0 + 64, head * kHeadDim, src + kOutBlockBytes);
                     }
-                    const int chunk = cb * 4 + c8;  // 16-byte chunk of the head vector: pairs 4 * chunk ..
-                    rope_rotate8(x, p.grid, pos, rope_chunk(p.grid, chunk));
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        out_of_range |= !(fabsf(x[i]) <= 65504.0f);
-                        if (!live || !ok) x[i] = 0.f;   // padding rows of K' are zero
-                    }
-                    uint4 w;
-                    w.x = pack_f16x2(x[0], x[1]);
-                    w.y = pack_f16x2(x[2], x[3]);
-                    w.z = pack_f16x2(x[4], x[5]);
-                    w.w = pack_f16x2(x[6], x[7]);
-                    const int col = cb * 32 + c8 * 8;
-                    *reinterpret_cast<uint4*>(stage_out + (col >> 6) * kOutBlockBytes + sw128_offset(row, (col >> 3) & 7)) = w;
                 }
+                tma_store_commit();
             }
-            if (out_of_range && live && ok) atomicCAS(p.status, 0, kStatusRange);
-        } else {
-            // v: row = feature of head `half`, columns = the tile's tokens
-            const float b = bias_s[half * 128 + row];
-#pragma unroll 1
-            for (int cb = 0; cb < 4; ++cb) {
-                uint32_t a[32];
-                if (ok) {
-                    tmem_ld32(t_acc + cb * 32, a);
-                    tmem_wait_ld();
-                }
-#pragma unroll
-                for (int c8 = 0; c8 < 4; ++c8) {
-                    float x[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int n = n0 + cb * 32 + c8 * 8 + i;
-                        x[i] = (ok && n < p.n_tokens) ? __uint_as_float(a[c8 * 8 + i]) + b : 0.f;  // padding columns zero
-                        out_of_range |= !(fabsf(x[i]) <= 65504.0f);
-                    }
-                    uint4 w;
-                    w.x = pack_f16x2(x[0], x[1]);
-                    w.y = pack_f16x2(x[2], x[3]);
-                    w.z = pack_f16x2(x[4], x[5]);
-                    w.w = pack_f16x2(x[6], x[7]);
-                    const int col = cb * 32 + c8 * 8;
-                    *reinterpret_cast<uint4*>(stage_out + (col >> 6) * kOutBlockBytes + sw128_offset(row, (col >> 3) & 7)) = w;
-                }
-            }
-            if (out_of_range) atomicCAS(p.status, 0, kStatusRange);
         }
-        fence_proxy_async_smem();
-        epi_barrier();
-        if (tid == 64 && ok) {
-#pragma unroll
-            for (int i = 0; i < kProjHeadsPerCta; ++i) {
-                const int head = pair * kProjHeadsPerCta + i;
-                const uint32_t src = smem_u32(stages + i * kOutTileBytes);
-                if (part == 0) {
-                    tma_store_2d(&tmap_q, head * kHeadDim, n0, src);
-                    tma_store_2d(&tmap_q, head * kHeadDim + 64, n0, src + kOutBlockBytes);
-                } else if (part == 1) {
-                    tma_store_2d(&tmap_k, 0, head * p.n_pad + n0, src);
-                    tma_store_2d(&tmap_k, 64, head * p.n_pad + n0, src + kOutBlockBytes);
-                } else {
-                    tma_store_2d(&tmap_v, n0, head * kHeadDim, src);
-                    tma_store_2d(&tmap_v, n0 + 64, head * kHeadDim, src + kOutBlockBytes);
-                }
-            }
-            tma_store_commit();
-            tma_store_wait_read();
-        }
+        if (tid == 64) tma_store_wait_read();
         __syncwarp();
     }
 
@@ -306,30 +423,29 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     __syncthreads();
     if (warp == 1) {
         __syncwarp();
-        if (bar->abort_flag) {
+        if (sh->abort_flag) {
             const uint64_t t0 = global_timer_ns();
             while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
         }
         __syncwarp();
-        tmem_dealloc(tmem_base, kFeat);
+        tmem_dealloc(tmem_base, 512);
     }
-    // no CTA of the cluster may exit while another can still read its row sums
-    if (normed) {
-        __syncwarp();
-        cluster_sync_all();
-    }
+    // no CTA of the cluster leaves while another could still write into its shared memory
+    __syncwarp();
+    cluster_sync_all();
 }
 
 cudaError_t configure_qkv_project() {
-    return cudaFuncSetAttribute(qkv_project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProjSmem);
+    cudaError_t e = cudaFuncSetAttribute(qkv_project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProjSmem);
+    return e;
 }
 
 cudaError_t launch_qkv_project(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w, const CUtensorMap& tmap_q,
                                const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const ProjParams& p,
-                               cudaStream_t stream) {
+                               int sm_count, cudaStream_t stream) {
     const unsigned cluster = p.h / kProjHeadsPerCta;
+    const int n_units = 3 * ((p.n_tokens + kTile - 1) / kTile);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cluster, (p.n_tokens + kTile - 1) / kTile, 3);
     cfg.blockDim = dim3(kProjThreads);
     cfg.dynamicSmemBytes = kProjSmem;
     cfg.stream = stream;
@@ -340,6 +456,19 @@ cudaError_t launch_qkv_project(const CUtensorMap& tmap_x, const CUtensorMap& tma
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    // one CTA per SM; as many clusters as can be resident at once (clusters do not straddle GPCs), at most one per unit
+    cfg.gridDim = dim3(cluster * (unsigned)(sm_count / (int)cluster > 0 ? sm_count / (int)cluster : 1));
+    // (asked once per cluster size; the GPUs of one process are taken to be alike)
+    static int resident[kProjMaxCluster + 1] = {};
+    int max_clusters = resident[cluster];
+    if (max_clusters == 0) {
+        cudaError_t e = cudaOccupancyMaxActiveClusters(&max_clusters, qkv_project_kernel, &cfg);
+        if (e != cudaSuccess) return e;
+        if (max_clusters < 1) return cudaErrorInvalidConfiguration;
+        resident[cluster] = max_clusters;
+    }
+    const int n_clusters = max_clusters < n_units ? max_clusters : n_units;
+    cfg.gridDim = dim3(cluster * (unsigned)n_clusters);
     return cudaLaunchKernelEx(&cfg, qkv_project_kernel, tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, p);
 }
 
