@@ -22,7 +22,7 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     return d;
 }
 
-__global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
+__global__ void __launch_bounds__(kPrepThreads, 4) prep_kv_kernel(PrepParams p) {
     const int tid = threadIdx.x;
     const int tile0 = blockIdx.x * kTile;
     const int head = blockIdx.y;
@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
     if (blockIdx.z == 0) {
         // ---- K: 16 threads per row (16 B = 8 elements = 4 rotary pairs each); all loads first
         const int chunk = tid & 15;
-        bool out_of_range = false;
+        float amax = 0.f;  // largest magnitude this thread writes (for the fp16 range check)
         __shared__ TokenPos s_pos[kTile];  // grid position of every row of the tile: one division pair per row
         uint4 raw[kTile / 16];
 #pragma unroll
@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
             bf16x8_to_float(raw[it], x);
             if (p.rope && n < p.n_kv) rope_rotate8(x, p.grid, s_pos[row], rc);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) out_of_range |= !(fabsf(x[i]) <= 65504.0f);
+            for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(x[i]));
             uint4 packed;
             packed.x = pack_f16x2(x[0], x[1]);
             packed.y = pack_f16x2(x[2], x[3]);
@@ -66,7 +66,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
             packed.w = pack_f16x2(x[6], x[7]);
             reinterpret_cast<uint4*>(p.kp + ((size_t)head * p.n_kv_pad + n) * kHeadDim)[chunk] = packed;
         }
-        if (out_of_range) atomicCAS(p.status, 0, kStatusRange);
+        if (!(amax <= 65504.0f)) atomicCAS(p.status, 0, kStatusRange);
     } else {
         // ---- V: transpose a [128 tokens][128 d] tile through shared memory.
         // tile[d][tp ^ swz(d)] holds the fp16 pair (token 2*tp, token 2*tp+1) of column d; swz(d) = (d / 4) % 32
@@ -74,7 +74,9 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
         __shared__ uint32_t tile[kHeadDim * 64];
         const int warp = tid >> 5, lane = tid & 31;
         const int tb = lane >> 4, c = lane & 15;  // token of the pair, 8-column chunk
-        bool out_of_range = false;
+        // |v| <= 65504 on the bf16 bit patterns: the largest bf16 not above 65504 is 0x477F (65280), so a 15-bit
+        // magnitude above it (Inf and NaN included) is out of range; checked two values per word with a running maximum
+        uint32_t mag_max = 0;
         uint4 raw[8];
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
@@ -88,8 +90,8 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
             const int tp = warp * 8 + it;
             float x[8];
             bf16x8_to_float(raw[it], x);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) out_of_range |= !(fabsf(x[i]) <= 65504.0f);
+            mag_max = __vmaxu2(mag_max, __vmaxu2(__vmaxu2(raw[it].x & 0x7fff7fffu, raw[it].y & 0x7fff7fffu),
+                                                 __vmaxu2(raw[it].z & 0x7fff7fffu, raw[it].w & 0x7fff7fffu)));
             const uint32_t h0 = pack_f16x2(x[0], x[1]), h1 = pack_f16x2(x[2], x[3]);
             const uint32_t h2 = pack_f16x2(x[4], x[5]), h3 = pack_f16x2(x[6], x[7]);
             // the lane of token 0 keeps columns 0..3 of the chunk, the lane of token 1 columns 4..7
@@ -105,7 +107,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kv_kernel(PrepParams p) {
             tile[(d0 + 2) * 64 + col] = prmt(lo_b, hi_b, 0x5410);
             tile[(d0 + 3) * 64 + col] = prmt(lo_b, hi_b, 0x7632);
         }
-        if (out_of_range) atomicCAS(p.status, 0, kStatusRange);
+        if ((mag_max & 0xffffu) > 0x477fu || (mag_max >> 16) > 0x477fu) atomicCAS(p.status, 0, kStatusRange);
         __syncthreads();
         uint32_t* dst = reinterpret_cast<uint32_t*>(p.vt + (size_t)head * kHeadDim * p.n_kv_pad + tile0);
         const size_t row_words = (size_t)p.n_kv_pad / 2;
