@@ -451,7 +451,7 @@ def run_ours(args, w: synth.Workload):
         # epilogue, followed by attention on those operands, against projection-then-attention (library GEMM and
         # element-wise kernels writing bf16 q, k, v, then the ordinary self-attention call)
         fusion = None
-        if not args.no_producer and w.n_heads % 2 == 0 and w.n_heads <= 16:
+        if not args.no_producer and w.n_heads % 2 == 0:
             fusion = time_producer_fusion(binding, w, dev, stream)
 
         # ---- end to end through the host-buffer entry points (pinned host memory, copies inside the timed region)

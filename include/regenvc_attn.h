@@ -139,10 +139,13 @@ int regenvc_attn_forward_prepared(const void* q_rot, const void* prepared, void*
  *   prepared : device, 256-byte aligned, regenvc_prepared_bytes(T*H*W, n_heads, 128) bytes: K' then V't (written,
  *              padding zero)
  * Arithmetic: bf16 products accumulated in fp32, norm and rotation in fp32, one rounding to fp16.  A result
- * beyond the fp16 range sets the sticky REGENVC_ERR_RANGE status.  n_heads must be even and at most 16 (the
- * n_heads / 2 thread blocks that share a token tile exchange their partial sums of squares as one cluster):
- * otherwise REGENVC_ERR_UNSUPPORTED.  Asynchronous on `stream`; allocates only the rotary table of a new
- * (T, H, W, theta).  Typical use:
+ * beyond the fp16 range sets the sticky REGENVC_ERR_RANGE status.  n_heads must be even (a thread block computes two
+ * heads of a token tile): otherwise REGENVC_ERR_UNSUPPORTED.  The thread blocks that share a token tile exchange
+ * their partial sums of squares through 6 * T*H*W * n_heads bytes (plus counters) of the calling thread's
+ * workspace -- regenvc_workspace_bytes(T*H*W, n_heads, 128) is always enough for a caller-supplied one -- and wait
+ * for each other with the same bounded waits as everything else (REGENVC_ERR_TIMEOUT if the GPU is shared with
+ * work that keeps part of the grid from becoming resident for half a second).  Asynchronous on `stream`; allocates
+ * only the rotary table of a new (T, H, W, theta) and, the first time, the workspace.  Typical use:
  *     regenvc_qkv_rope_project(x, w, b, gq, gk, eps, q_rot, prepared, T, H, W, h, 128, theta, s);
  *     regenvc_attn_forward_prepared(q_rot, prepared, out, T*H*W, T*H*W, h, 128, s);
  */

@@ -584,8 +584,7 @@ int regenvc_qkv_rope_project(const void* x, const void* w_qkv, const void* b_qkv
     if (n_heads < 1 || head_dim < 1) return REGENVC_ERR_BAD_SHAPE;
     const long long n_pad = (n + kTile - 1) / kTile * kTile;
     if (n_heads > 65535 || n_pad * n_heads >= (1ll << 31)) return REGENVC_ERR_BAD_SHAPE;
-    if (head_dim != kHeadDim || n_heads % kProjHeadsPerCta != 0 || n_heads / kProjHeadsPerCta > kProjMaxCluster)
-        return REGENVC_ERR_UNSUPPORTED;
+    if (head_dim != kHeadDim || n_heads % kProjHeadsPerCta != 0) return REGENVC_ERR_UNSUPPORTED;
     if (!(rope_theta > 0.0f) || !std::isfinite(rope_theta) || !(eps >= 0.0f) || !std::isfinite(eps))
         return REGENVC_ERR_UNSUPPORTED;
     if (((uintptr_t)x | (uintptr_t)w_qkv | (uintptr_t)q_rot | (uintptr_t)b_qkv | (uintptr_t)g_q | (uintptr_t)g_k) & 15)
@@ -602,7 +601,24 @@ int regenvc_qkv_rope_project(const void* x, const void* w_qkv, const void* b_qkv
     DeviceState* st = nullptr;
     rc = device_state(&dev, &st);
     if (rc != REGENVC_OK) return rc;
+    // scratch for the norm's sums: the caller's workspace if one is set, else this thread's own
+    const size_t need = proj_scratch_bytes(n, n_heads);
+    char* ws = nullptr;
+    Workspace* own = nullptr;
+    if (tl_user_ws.ptr) {
+        if (tl_user_ws.bytes < need) return REGENVC_ERR_WORKSPACE;
+        ws = reinterpret_cast<char*>(tl_user_ws.ptr);
+    } else {
+        own = &st->workspace[std::this_thread::get_id()];
+        rc = grow(own->buf, need);
+        if (rc != REGENVC_OK) return rc;
+        ws = reinterpret_cast<char*>(own->buf.ptr);
+        rc = order_after_last_user(*own, (cudaStream_t)stream);
+        if (rc != REGENVC_OK) return rc;
+    }
     ProjParams pp;
+    pp.unit_count = reinterpret_cast<int*>(ws);
+    pp.unit_sums = reinterpret_cast<float*>(ws + proj_count_bytes(n));
     pp.bias = reinterpret_cast<const float*>(b_qkv);
     pp.g_q = reinterpret_cast<const float*>(g_q);
     pp.g_k = reinterpret_cast<const float*>(g_k);
@@ -629,7 +645,7 @@ int regenvc_qkv_rope_project(const void* x, const void* w_qkv, const void* b_qkv
     if (rc != REGENVC_OK) return rc;
     CUDA_TRY(launch_qkv_project(tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, pp, st->sm_count, (cudaStream_t)stream));
     launched();
-    return REGENVC_OK;
+    return own ? note_use(*own, (cudaStream_t)stream) : REGENVC_OK;
 }
 
 int regenvc_attn_forward_host(const void* q, const void* k, const void* v, void* out, int T, int H, int W, int n_heads,

@@ -69,7 +69,6 @@ struct AttnParams {
 
 // QKV projection with fused norm / rotation / operand-layout epilogue (producer of the attention operands).
 constexpr int kProjHeadsPerCta = 2;   // a CTA computes 128 tokens x two heads of one of q, k, v per work unit
-constexpr int kProjMaxCluster = 8;    // the CTAs that share a token tile form one cluster (h / 2 of them)
 struct ProjParams {
     const float* bias;        // [3C] or nullptr
     const float* g_q;         // [C] RMS-norm gains of q (nullptr: ones)
@@ -78,7 +77,20 @@ struct ProjParams {
     int n_tokens, n_pad, C, h;
     RopeGrid grid;
     int* status;
+    // scratch of the norm's sum over all features: per (128-token tile, q/k/v) unit one counter of the slices that
+    // have published their partial row sums, and the sums themselves [unit][slice][128 tokens]
+    int* unit_count;
+    float* unit_sums;
 };
+// Bytes of that scratch for n_tokens tokens and h heads (counters first, 256-byte aligned, then the sums).
+inline size_t proj_count_bytes(long long n_tokens) {
+    const size_t n_units = 3 * (size_t)((n_tokens + kTile - 1) / kTile);
+    return (n_units * sizeof(int) + 255) / 256 * 256;
+}
+inline size_t proj_scratch_bytes(long long n_tokens, int h) {
+    const size_t n_units = 3 * (size_t)((n_tokens + kTile - 1) / kTile);
+    return proj_count_bytes(n_tokens) + n_units * (size_t)(h / kProjHeadsPerCta) * kTile * sizeof(float);
+}
 cudaError_t configure_qkv_project();
 cudaError_t launch_qkv_project(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w, const CUtensorMap& tmap_q,
                                const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const ProjParams& p,

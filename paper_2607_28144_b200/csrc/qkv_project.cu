@@ -7,8 +7,9 @@
 //   V't fp16 [h][128][n_pad]      values, keys contiguous       } so no separate preparation pass is needed
 // and nothing of q, k, v is ever rounded to bf16 or written in token-major form.
 //
-// A work unit is (128-token tile, one of q / k / v); the h/2 CTAs of a thread-block cluster compute it together,
-// each 256 output features (two heads).  Clusters are persistent: cluster c takes units c, c + n_clusters, ...
+// A work unit is (128-token tile, one of q / k / v), cut into h/2 slices of 256 output features (two heads).  The
+// grid is persistent, one CTA per SM: CTA c takes slices c, c + gridDim.x, ... of the unit-major list, so the
+// slices of a unit run on neighbouring CTAs at about the same time.
 //   warp 0      TMA producer: x tile [128 tokens][64] and W tile [256 features][64] per stage (bf16, 128B swizzle),
 //               a 3-stage ring that runs on into the next unit
 //   warp 1      tcgen05.mma issuer (bf16 x bf16 -> fp32) and TMEM owner; two accumulators of 256 columns, used in
@@ -16,9 +17,14 @@
 //   warps 2-9   epilogue, two threads per accumulator row (one per head)
 // q and k: D[token][feature] = x W^T (A = x tile, B = W tile, N = 256).  v: D[feature][token] = W x^T (A = W rows of
 // one head, B = x tile), which is V't directly -- no transpose anywhere.
-// The RMS norm needs the sum of squares over ALL features of a token, which are spread over the CTAs of the cluster:
-// every CTA writes its partial row sums into the shared memory of all of them (distributed shared memory) and
-// arrives on their barriers; only the epilogue warps wait for it, the producer and the MMA warp run ahead.
+// The RMS norm needs the sum of squares over ALL features of a token, which are spread over the h/2 CTAs that hold
+// the slices of the unit: each writes its partial row sums to a scratch array in global memory and counts itself in
+// on the unit's counter; the epilogue warps (only they -- the producer and the MMA warp run ahead) wait until the
+// counter shows all slices and add the partial sums in slice order, so the result does not depend on timing.  The
+// wait is bounded like every other; it cannot deadlock because every CTA works through its slices in increasing
+// order and the whole grid is resident (grid <= number of SMs, one CTA per SM).  (A first form exchanged the sums
+// through distributed shared memory inside clusters of h/2 CTAs; clusters of 6 left 16 of this part's 148 SMs idle
+// and capped the head count at 16.)
 #include <cstddef>
 
 #include "common.cuh"
@@ -49,83 +55,22 @@ struct ProjShared {
     uint64_t empty[kProjStages];
     uint64_t acc_full[2];      // accumulator b holds a finished unit
     uint64_t acc_empty[2];     // the epilogue has read accumulator b out
-    uint64_t sums_in[2];       // every CTA of the cluster has delivered its partial row sums into xsum[b]
     uint32_t tmem_base;
     int abort_flag;
     float bias[kFeat];         // this unit's slice of the bias
     float gain[kFeat];         //             ... and of the norm gains
     float part[2][kTile];      // partial sums of squares of the two heads of this CTA
-    float xsum[2][kProjMaxCluster][kTile];  // [buffer][source CTA][token]: partial row sums of the whole cluster
 };
 constexpr uint32_t kProjSmem = kProjStages * kStageBytes + kProjHeadsPerCta * kOutTileBytes + 1024 /*align*/ +
                                sizeof(ProjShared);
 static_assert(kProjSmem <= 232448, "shared memory of one SM");
 
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t cluster_size() {
-    uint32_t n;
-    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(n));
-    return n;
-}
-__device__ __forceinline__ uint32_t cluster_rank() {
-    uint32_t n;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(n));
-    return n;
-}
-__device__ __forceinline__ uint32_t cluster_id_x() {
-    uint32_t n;
-    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(n));
-    return n;
-}
-__device__ __forceinline__ uint32_t n_clusters_x() {
-    uint32_t n;
-    asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(n));
-    return n;
-}
-// Address of the same shared-memory location in CTA `rank` of this cluster.
-__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    return remote;
-}
-// Asynchronous 4-byte store into the shared memory of a CTA of the cluster that counts its bytes on a barrier of that
-// same CTA: whoever sees the barrier's phase complete (acquire at cluster scope) sees the value.  No fence is needed
-// on the sending side (a release-arrive per store, tried first, cost about 1.7 k clocks each).
-__device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float v, uint32_t cluster_bar) {
-    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
-                 ::"r"(cluster_addr), "r"(__float_as_uint(v)), "r"(cluster_bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, const WaitCtl& ctl) {
-    uint64_t t0 = 0;
-    uint32_t spins = 0;
-    while (!mbar_try_wait_cluster(bar, parity)) {
-        if ((++spins & 255u) == 0) {
-            if (*ctl.abort_flag) return false;
-            const uint64_t now = global_timer_ns();
-            if (t0 == 0) {
-                t0 = now;
-            } else if (now - t0 > ctl.limit_ns) {
-                *ctl.abort_flag = 1;
-                atomicCAS(ctl.status, 0, ctl.code);
-                return false;
-            }
-        }
-    }
-    return true;
+// Value of a counter in global memory as other CTAs have left it (acquire at device scope).
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 
 }  // namespace
@@ -141,11 +86,10 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     ProjShared* sh = reinterpret_cast<ProjShared*>(stage_out + kProjHeadsPerCta * kOutTileBytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int pair = static_cast<int>(cluster_rank());       // which two heads
-    const int n_rank = static_cast<int>(cluster_size());
+    const int n_rank = p.h / kProjHeadsPerCta;               // slices per unit
     const int n_tiles = (p.n_tokens + kTile - 1) / kTile;
-    const int n_units = 3 * n_tiles;                         // unit u: token tile u / 3, part u % 3 (0 q, 1 k, 2 v)
-    const int unit0 = static_cast<int>(cluster_id_x()), unit_step = static_cast<int>(n_clusters_x());
+    const int n_slices = 3 * n_tiles * n_rank;               // slice s: unit s / n_rank (token tile unit / 3, part unit % 3:
+    const int slice0 = blockIdx.x, slice_step = gridDim.x;   // 0 q, 1 k, 2 v), heads 2 (s % n_rank) and 2 (s % n_rank) + 1
     const int n_kb = p.C / kBK;
     const WaitCtl ctl{&sh->abort_flag, p.status, kStatusTimeout, kProjWaitNs};
     uint32_t tmem_base = 0;
@@ -158,7 +102,6 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&sh->acc_full[b]), 1);
             mbar_init(smem_u32(&sh->acc_empty[b]), kEpiThreads);
-            mbar_init(smem_u32(&sh->sums_in[b]), 1);   // one local arrival that announces the bytes, then the bytes
         }
         sh->abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0) ? 1 : 0;
         fence_mbar_init();
@@ -170,8 +113,6 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     }
     tc_fence_before();
     __syncthreads();
-    // nobody may arrive on a barrier of another CTA before that CTA has initialised it
-    cluster_sync_all();
     tc_fence_after();
     tmem_base = sh->tmem_base;
 
@@ -182,9 +123,10 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             tma_prefetch_desc(&tmap_w);
             int fill = 0;  // stages filled so far over all units
             bool ok = true;
-            for (int unit = unit0; ok && unit < n_units; unit += unit_step) {
+            for (int slice = slice0; ok && slice < n_slices; slice += slice_step) {
+                const int unit = slice / n_rank, pair = slice % n_rank;
                 const int n0 = (unit / 3) * kTile;
-                const int f0 = (unit % 3) * p.C + pair * kFeat;   // first row of W_qkv (output feature) of this CTA
+                const int f0 = (unit % 3) * p.C + pair * kFeat;   // first row of W_qkv (output feature) of this slice
                 for (int kb = 0; kb < n_kb; ++kb, ++fill) {
                     const int s = fill % kProjStages, round = fill / kProjStages;
                     if (round > 0) ok = mbar_wait(smem_u32(&sh->empty[s]), (round - 1) & 1, ctl);
@@ -202,8 +144,8 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         if (elect_one()) {
             int fill = 0, it = 0;
             bool ok = true;
-            for (int unit = unit0; ok && unit < n_units; unit += unit_step, ++it) {
-                const int part = unit % 3, b = it & 1;
+            for (int slice = slice0; ok && slice < n_slices; slice += slice_step, ++it) {
+                const int part = (slice / n_rank) % 3, b = it & 1;
                 const uint32_t acc_tmem = tmem_base + b * kFeat;
                 // the accumulator must have been read out by the epilogue of the unit before last
                 if (it >= 2) ok = mbar_wait(smem_u32(&sh->acc_empty[b]), ((it >> 1) - 1) & 1, ctl);
@@ -240,8 +182,9 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         const int et = tid - 64;                      // 0 .. 255
         uint8_t* my_stage = stage_out + half * kOutTileBytes;
         bool ok = true;
-        int it = 0, normed_seen = 0;
-        for (int unit = unit0; unit < n_units; unit += unit_step, ++it) {
+        int it = 0;
+        for (int slice = slice0; slice < n_slices; slice += slice_step, ++it) {
+            const int unit = slice / n_rank, pair = slice % n_rank;
             const int part = unit % 3, n0 = (unit / 3) * kTile, b = it & 1;
             const bool normed = part < 2;
             const uint32_t t_acc = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + b * kFeat + half * 128;
@@ -277,20 +220,36 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 }
                 sh->part[half][row] = ss;
                 epi_barrier();
-                const int xb = normed_seen & 1;
-                if (et == 0) mbar_expect_tx(smem_u32(&sh->sums_in[xb]), n_rank * kTile * 4);  // what this CTA will receive
-                if (half == 0) {
-                    // deliver this CTA's partial sum of the token to every CTA of the cluster (itself included)
-                    const float mine = sh->part[0][row] + sh->part[1][row];
-                    const uint32_t slot = smem_u32(&sh->xsum[xb][pair][row]), barx = smem_u32(&sh->sums_in[xb]);
-                    for (int r = 0; r < n_rank; ++r) st_async_f32(map_to_rank(slot, r), mine, map_to_rank(barx, r));
+                // publish this slice's partial sum of every token, then count the slice in
+                if (half == 0)
+                    __stcg(p.unit_sums + ((size_t)unit * n_rank + pair) * kTile + row, sh->part[0][row] + sh->part[1][row]);
+                __threadfence();
+                epi_barrier();
+                if (et == 0) {
+                    atomicAdd(p.unit_count + unit, 1);
+                    uint64_t t0 = 0;
+                    uint32_t spins = 0;
+                    while (ok && ld_acquire_gpu(p.unit_count + unit) < n_rank) {   // all slices of the unit are in?
+                        __nanosleep(64);
+                        if ((++spins & 63u) == 0) {
+                            if (sh->abort_flag) ok = false;
+                            const uint64_t now = global_timer_ns();
+                            if (t0 == 0) t0 = now;
+                            else if (now - t0 > kProjWaitNs) {
+                                sh->abort_flag = 1;
+                                atomicCAS(p.status, 0, kStatusTimeout);
+                                ok = false;
+                            }
+                        }
+                    }
                 }
-                if (ok) ok = mbar_wait_cluster(smem_u32(&sh->sums_in[xb]), (normed_seen >> 1) & 1, ctl);
+                epi_barrier();
+                if (sh->abort_flag) ok = false;
                 ok = __all_sync(0xffffffffu, ok);
                 float total = 0.f;
-                for (int r = 0; r < n_rank; ++r) total += sh->xsum[xb][r][row];
+                for (int r = 0; r < n_rank; ++r)   // slice order: the same sum whatever the timing
+                    total += __ldcg(p.unit_sums + ((size_t)unit * n_rank + r) * kTile + row);
                 inv_rms = rsqrtf(total / static_cast<float>(p.C) + p.eps);
-                ++normed_seen;
             }
 
             // the staging tiles are free once the previous unit's stores have read them (thread 64 issued them)
@@ -430,9 +389,6 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         __syncwarp();
         tmem_dealloc(tmem_base, 512);
     }
-    // no CTA of the cluster leaves while another could still write into its shared memory
-    __syncwarp();
-    cluster_sync_all();
 }
 
 cudaError_t configure_qkv_project() {
@@ -443,33 +399,15 @@ cudaError_t configure_qkv_project() {
 cudaError_t launch_qkv_project(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w, const CUtensorMap& tmap_q,
                                const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const ProjParams& p,
                                int sm_count, cudaStream_t stream) {
-    const unsigned cluster = p.h / kProjHeadsPerCta;
     const int n_units = 3 * ((p.n_tokens + kTile - 1) / kTile);
-    cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(kProjThreads);
-    cfg.dynamicSmemBytes = kProjSmem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cluster;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    // one CTA per SM; as many clusters as can be resident at once (clusters do not straddle GPCs), at most one per unit
-    cfg.gridDim = dim3(cluster * (unsigned)(sm_count / (int)cluster > 0 ? sm_count / (int)cluster : 1));
-    // (asked once per cluster size; the GPUs of one process are taken to be alike)
-    static int resident[kProjMaxCluster + 1] = {};
-    int max_clusters = resident[cluster];
-    if (max_clusters == 0) {
-        cudaError_t e = cudaOccupancyMaxActiveClusters(&max_clusters, qkv_project_kernel, &cfg);
-        if (e != cudaSuccess) return e;
-        if (max_clusters < 1) return cudaErrorInvalidConfiguration;
-        resident[cluster] = max_clusters;
-    }
-    const int n_clusters = max_clusters < n_units ? max_clusters : n_units;
-    cfg.gridDim = dim3(cluster * (unsigned)n_clusters);
-    return cudaLaunchKernelEx(&cfg, qkv_project_kernel, tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, p);
+    const int n_slices = n_units * (p.h / kProjHeadsPerCta);
+    // the counters of the units start at zero; the partial sums need no clearing (every slot is written before read)
+    cudaError_t e = cudaMemsetAsync(p.unit_count, 0, (size_t)n_units * sizeof(int), stream);
+    if (e != cudaSuccess) return e;
+    // one CTA per SM and never more CTAs than SMs: the whole grid is resident, which the waits between slices rely on
+    const int grid = n_slices < sm_count ? n_slices : sm_count;
+    qkv_project_kernel<<<grid, kProjThreads, kProjSmem, stream>>>(tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, p);
+    return cudaGetLastError();
 }
 
 }  // namespace regenvc
