@@ -66,7 +66,10 @@ typedef enum {
     REGENVC_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired (sticky device status) */
     REGENVC_ERR_WORKSPACE = 8,   /* caller-supplied workspace too small or misaligned */
     REGENVC_ERR_RANGE = 9,       /* an input exceeded the fp16 operand range (sticky device status) */
-    REGENVC_ERR_STATIC_LIMIT = 10 /* regenvc_cross_attn_forward_static(): the shape needs more than the built-in scratch */
+    REGENVC_ERR_STATIC_LIMIT = 10, /* regenvc_cross_attn_forward_static(): the shape needs more than the built-in scratch */
+    REGENVC_ERR_INTERNAL = 11     /* a kernel found an assumption about its launch broken and did no work (sticky device
+                                     status): the dynamic shared memory of the persistent attention kernel did not
+                                     start on a 1024-byte boundary */
 } regenvc_status;
 
 /*

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libregenvc_attn.so")
 
 OK, ERR_NULL_POINTER, ERR_BAD_SHAPE, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_ALIASING, ERR_CUDA, ERR_TIMEOUT, \
-    ERR_WORKSPACE, ERR_RANGE, ERR_STATIC_LIMIT = range(11)
+    ERR_WORKSPACE, ERR_RANGE, ERR_STATIC_LIMIT, ERR_INTERNAL = range(12)
 STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = [

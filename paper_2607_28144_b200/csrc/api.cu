@@ -880,6 +880,7 @@ const char* regenvc_status_string(int status) {
         case REGENVC_ERR_WORKSPACE: return "workspace too small or misaligned";
         case REGENVC_ERR_RANGE: return "input outside the fp16 operand range";
         case REGENVC_ERR_STATIC_LIMIT: return "shape exceeds the built-in scratch of the allocation-free entry point";
+        case REGENVC_ERR_INTERNAL: return "a kernel found its launch assumptions broken and did no work";
         default: return "unknown status";
     }
 }

@@ -101,7 +101,7 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = smem_raw;
     if ((smem_u32(base) & 1023u) != 0) {  // the swizzled tiles need a 1024-byte aligned base (uniform over the grid)
-        if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusTimeout);
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, kStatusInternal);
         return;
     }
     uint8_t* sQ = base;                                   // 2 tiles

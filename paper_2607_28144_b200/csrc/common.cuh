@@ -17,6 +17,7 @@ constexpr int kPairsX = 21;         // x axis (width 42)
 // Sticky device status codes (mirror regenvc_status).
 constexpr int kStatusTimeout = 7;
 constexpr int kStatusRange = 9;
+constexpr int kStatusInternal = 11;
 
 // cos/sin table of one (T, H, W, theta): float2 (cos, sin) entries,
 // [T][22] then [H][21] then [W][21].

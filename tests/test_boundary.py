@@ -35,8 +35,8 @@ def test_every_declared_symbol_is_exported(L):
 
 def test_status_strings_and_version(L):
     assert binding.regenvc_version().startswith("regenvc-attn")
-    seen = {binding.status_string(c) for c in range(11)}
-    assert len(seen) == 11 and binding.status_string(99) == "unknown status"
+    seen = {binding.status_string(c) for c in range(12)}
+    assert len(seen) == 12 and binding.status_string(99) == "unknown status"
 
 
 def test_workspace_bytes():
