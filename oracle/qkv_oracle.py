@@ -15,6 +15,13 @@ GPU path that fuses these steps into the projection's epilogue is compared with 
 
 The weights are stored the way a linear layer stores them: w_qkv [3C, C], row f holds the weights of output
 feature f; rows 0..C-1 make y_q, C..2C-1 make y_k, 2C..3C-1 make v.  b_qkv [3C], g_q, g_k [C].
+
+The step behind the attention in the same block is its output projection: the heads' outputs of a token, laid side
+by side as one row of C features (head a in features a*head_dim ...), go through one more linear map,
+
+    y = o W_o^T + b_o                                                         (C -> C),
+
+written out in `out_project`; `attention_block` chains all three steps without rounding anything in between.
 """
 from __future__ import annotations
 
@@ -68,3 +75,24 @@ def projected_self_attention(x_bits, w_bits, b, g_q, g_k, eps, n_heads, T, H, W,
     """Projection, norm, rotation and exact softmax attention; fp64 [n_rows, n_heads_listed, d]."""
     ops = rotated_operands(x_bits, w_bits, b, g_q, g_k, eps, n_heads, T, H, W, theta, heads)
     return np.stack([_o.attn_core_head(qr, kr, v, rows) for qr, kr, v in ops.values()], axis=1)
+
+
+def out_project(o_bits, w_o_bits, b_o) -> np.ndarray:
+    """o [N, C] (the attention output, heads side by side) and w_o [C_out, C] as bf16 bit patterns, b_o [C_out]
+    float or None.  Returns y = o w_o^T + b_o as fp64 [N, C_out]."""
+    o, w = bf16_to_f64(o_bits), bf16_to_f64(w_o_bits)
+    o = o.reshape(o.shape[0], -1)
+    if w.ndim != 2 or w.shape[1] != o.shape[1]:
+        raise ValueError("w_o must be [C_out, C] with C the feature count of o")
+    b = np.zeros(w.shape[0]) if b_o is None else np.asarray(b_o, dtype=np.float64)
+    return o @ w.T + b[None, :]
+
+
+def attention_block(x_bits, w_bits, b, g_q, g_k, eps, n_heads, T, H, W, w_o_bits, b_o, theta=10000.0,
+                    rows=None) -> np.ndarray:
+    """The whole attention part of a block in fp64, nothing rounded between the steps: projection, norm, rotation,
+    exact softmax attention over all heads, output projection.  Returns y [n_rows, C_out]."""
+    o = projected_self_attention(x_bits, w_bits, b, g_q, g_k, eps, n_heads, T, H, W, theta, rows)
+    w = bf16_to_f64(w_o_bits)
+    bo = np.zeros(w.shape[0]) if b_o is None else np.asarray(b_o, dtype=np.float64)
+    return o.reshape(o.shape[0], -1) @ w.T + bo[None, :]

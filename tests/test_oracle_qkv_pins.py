@@ -131,3 +131,43 @@ def test_query_gain_acts_as_a_softmax_temperature_and_rows_subset_matches():
     full = qo.projected_self_attention(x, w, b, gq, gk, 1e-6, h, T, H, W)
     part = qo.projected_self_attention(x, w, b, gq, gk, 1e-6, h, T, H, W, rows=rows, heads=[1])
     np.testing.assert_array_equal(part[:, 0], full[rows, 1])
+
+
+def test_output_projection_against_plain_loops_and_its_special_cases():
+    """Every element by scalar loops (catches a transposed weight and a bias added per token instead of per
+    feature); the identity returns its input; a permutation matrix permutes features; zero weights leave the bias."""
+    N, C, Co = 3, 8, 5
+    rng = np.random.default_rng(7)
+    o = _bits(rng.integers(-6, 7, (N, 2, C // 2)) / 4.0)      # two heads of four features, side by side
+    w = _bits(rng.integers(-4, 5, (Co, C)) / 8.0)
+    b = rng.integers(-3, 4, Co) / 4.0
+    y = qo.out_project(o, w, b)
+    of, wf = qo.bf16_to_f64(o).reshape(N, C), qo.bf16_to_f64(w)
+    assert y.shape == (N, Co)
+    for n in range(N):
+        for f in range(Co):
+            assert y[n, f] == pytest.approx(sum(of[n, c] * wf[f, c] for c in range(C)) + b[f], rel=1e-14, abs=1e-15)
+    np.testing.assert_array_equal(qo.out_project(o, _bits(np.eye(C)), None), of)
+    perm = rng.permutation(C)
+    np.testing.assert_array_equal(qo.out_project(o, _bits(np.eye(C)[perm]), None), of[:, perm])
+    np.testing.assert_array_equal(qo.out_project(o, _bits(np.zeros((Co, C))), b), np.broadcast_to(b, (N, Co)))
+
+
+def test_attention_block_reduces_to_its_parts():
+    """With W_o = I and no bias the block is the projected self-attention with the heads laid side by side; in
+    general it is out_project applied to that result (checked with values that survive the bf16 round trip:
+    one-hot W_o rows pick single features, so nothing is rounded)."""
+    T, H, W, h = 1, 3, 4, 2
+    N, C = T * H * W, h * D
+    x, w, b, gq, gk = _setup(N, h, 8)
+    att = qo.projected_self_attention(x, w, b, gq, gk, 1e-6, h, T, H, W)
+    blk = qo.attention_block(x, w, b, gq, gk, 1e-6, h, T, H, W, _bits(np.eye(C)), None)
+    np.testing.assert_array_equal(blk, att.reshape(N, C))
+    rng = np.random.default_rng(9)
+    pick = rng.integers(0, C, size=7)
+    sel = np.zeros((7, C))
+    sel[np.arange(7), pick] = 2.0
+    bo = rng.standard_normal(7)
+    rows = [0, 3, N - 1]
+    blk = qo.attention_block(x, w, b, gq, gk, 1e-6, h, T, H, W, _bits(sel), bo, rows=rows)
+    np.testing.assert_allclose(blk, 2.0 * att.reshape(N, C)[rows][:, pick] + bo[None, :], rtol=1e-14, atol=1e-15)
