@@ -269,7 +269,16 @@ def time_producer_fusion(binding, w: synth.Workload, dev, stream, n=20):
         torch.cuda.synchronize()
         return statistics.mean(a.elapsed_time(bb) for a, bb in evs)
 
+    wo, bo = (t.to(dev) for t in synth.out_proj_inputs(w))
+    y = torch.empty((N, C), dtype=torch.bfloat16, device=dev)
+    bo16 = bo.to(torch.bfloat16)
+    out2d = out.view(N, C)
+
+    def out_proj():
+        binding.regenvc_out_project(out, wo, bo, y=y, stream=stream)
+
     t_prod, t_attn_p = timed(producer), timed(attn_prepared)
+    t_oproj, t_oproj_lib = timed(out_proj), timed(lambda: torch.addmm(bo16, out2d, wo.t()))
     t_gemm = timed(lambda: torch.addmm(b16, x, wq.t()))
     t_lib, t_attn = timed(library_projection), timed(attn_plain)
     flops = 2.0 * N * 3 * C * C
@@ -277,8 +286,11 @@ def time_producer_fusion(binding, w: synth.Workload, dev, stream, n=20):
             "attention_on_prepared_operands_ms": t_attn_p, "fused_ms": t_prod + t_attn_p,
             "library_gemm_only_ms": t_gemm, "library_projection_norm_ms": t_lib,
             "attention_with_preparation_pass_ms": t_attn, "unfused_ms": t_lib + t_attn,
+            "out_project_ms": t_oproj, "out_project_tflops": 2.0 * N * C * C / (t_oproj * 1e-3) / 1e12,
+            "library_out_project_gemm_ms": t_oproj_lib, "block_attention_part_ms": t_prod + t_attn_p + t_oproj,
             "note": "fused = regenvc_qkv_rope_project + regenvc_attn_forward_prepared (no preparation pass, no "
-                    "bf16 round trip of q, k, v); unfused = library GEMM + eager norm kernels + regenvc_attn_forward"}
+                    "bf16 round trip of q, k, v); unfused = library GEMM + eager norm kernels + regenvc_attn_forward; "
+                    "block_attention_part = fused + regenvc_out_project (y = o W_o^T + b_o, bf16)"}
 
 
 def run_ours(args, w: synth.Workload):

@@ -159,6 +159,21 @@ int regenvc_qkv_rope_project(const void* x, const void* w_qkv, const void* b_qkv
                              float rope_theta, void* stream);
 
 /*
+ * The step behind the attention in the same block (backbone by reference, Sec. 3.2 / 3.4): its output projection
+ *     y = o W_o^T + b_o
+ * on the attention output exactly as the attention entry points leave it (the heads of a token side by side are
+ * one row of C = n_heads * 128 features), with the bias and the rounding to bf16 in the epilogue:
+ *   attn_out : device, bf16 [n_tokens, n_heads, 128]                           (read only)
+ *   w_o      : device, bf16 [C, C]; row f = weights of output feature f
+ *   b_o      : device, fp32 [C], or NULL for no bias
+ *   y        : device, bf16 [n_tokens, C]                (written; must not overlap the inputs)
+ * Arithmetic: bf16 products accumulated in fp32, bias added in fp32, one rounding to bf16.  n_heads must be even
+ * (REGENVC_ERR_UNSUPPORTED otherwise).  No workspace, no allocation, asynchronous on `stream`.
+ */
+int regenvc_out_project(const void* attn_out, const void* w_o, const void* b_o, void* y,
+                        int n_tokens, int n_heads, int head_dim, void* stream);
+
+/*
  * Block-wise attention for sequence-parallel use (Sec. 3.5: Ring attention streams key/value blocks around
  * the devices and combines the per-block results by the online-softmax rule; the result is unsharded
  * attention, only summed in another order).

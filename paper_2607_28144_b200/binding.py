@@ -26,7 +26,7 @@ EXPORTS = [
     "regenvc_kernel_launch_count", "regenvc_shutdown", "regenvc_debug_set_phases",
     "regenvc_cross_attn_forward_static", "regenvc_static_device_status", "regenvc_attn_partial",
     "regenvc_prepared_bytes", "regenvc_cross_kv_prepare", "regenvc_cross_attn_forward_prepared",
-    "regenvc_attn_forward_prepared", "regenvc_qkv_rope_project", "regenvc_attn_merge",
+    "regenvc_attn_forward_prepared", "regenvc_qkv_rope_project", "regenvc_out_project", "regenvc_attn_merge",
     "regenvc_ulysses_scatter_heads", "regenvc_ulysses_gather_heads", "regenvc_debug_expire_wait",
 ]
 
@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
     L.regenvc_attn_forward_prepared.restype = i32
     L.regenvc_qkv_rope_project.argtypes = [vp, vp, vp, vp, vp, f32, vp, vp, i32, i32, i32, i32, i32, f32, vp]
     L.regenvc_qkv_rope_project.restype = i32
+    L.regenvc_out_project.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
+    L.regenvc_out_project.restype = i32
     L.regenvc_workspace_bytes.argtypes = [i32, i32, i32]
     L.regenvc_workspace_bytes.restype = sz
     L.regenvc_set_workspace.argtypes = [vp, sz]
@@ -236,6 +238,25 @@ def regenvc_qkv_rope_project(x, w_qkv, b_qkv, g_q, g_k, eps: float, T: int, H: i
                                           q_rot.data_ptr(), prepared.data_ptr(), T, H, W, n_heads, 128,
                                           float(rope_theta), _stream(stream)))
     return q_rot, prepared
+
+
+def regenvc_out_project(attn_out, w_o, b_o, y=None, stream=None):
+    """Output projection of the block: attn_out CUDA bf16 [tokens, heads, 128] (as the attention calls write it),
+    w_o CUDA bf16 [C, C], b_o CUDA fp32 [C] or None.  Returns y bf16 [tokens, C] (allocated with torch if not given)."""
+    _dev_bf16(attn_out, "attn_out")
+    n, h, d = attn_out.shape
+    C = h * d
+    if w_o.dtype != torch.bfloat16 or not w_o.is_cuda or not w_o.is_contiguous() or tuple(w_o.shape) != (C, C):
+        raise TypeError("w_o must be a contiguous CUDA bf16 tensor [C, C]")
+    if b_o is not None and (b_o.dtype != torch.float32 or not b_o.is_cuda or not b_o.is_contiguous() or b_o.numel() != C):
+        raise TypeError(f"b_o must be a contiguous CUDA fp32 tensor of {C} elements (or None)")
+    if y is None:
+        y = torch.empty((n, C), dtype=torch.bfloat16, device=attn_out.device)
+    if y.dtype != torch.bfloat16 or not y.is_cuda or not y.is_contiguous() or tuple(y.shape) != (n, C):
+        raise TypeError("y must be a contiguous CUDA bf16 tensor [tokens, C]")
+    _check(lib().regenvc_out_project(attn_out.data_ptr(), w_o.data_ptr(), None if b_o is None else b_o.data_ptr(),
+                                     y.data_ptr(), n, h, d, _stream(stream)))
+    return y
 
 
 def regenvc_cross_attn_forward_static(q, k, v, out, stream=None):

@@ -124,6 +124,7 @@ int device_state(int* dev_out, DeviceState** st_out) {
             }
             CUDA_TRY(configure_attn_pipelined());
             CUDA_TRY(configure_qkv_project());
+            CUDA_TRY(configure_out_project());
             CUDA_TRY(configure_attn_persistent());
             CUDA_TRY(cudaMalloc(&st.status, sizeof(int)));
             CUDA_TRY(cudaMemset(st.status, 0, sizeof(int)));
@@ -646,6 +647,42 @@ int regenvc_qkv_rope_project(const void* x, const void* w_qkv, const void* b_qkv
     CUDA_TRY(launch_qkv_project(tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, pp, st->sm_count, (cudaStream_t)stream));
     launched();
     return own ? note_use(*own, (cudaStream_t)stream) : REGENVC_OK;
+}
+
+int regenvc_out_project(const void* attn_out, const void* w_o, const void* b_o, void* y, int n_tokens,
+                        int n_heads, int head_dim, void* stream) {
+    if (!attn_out || !w_o || !y) return REGENVC_ERR_NULL_POINTER;
+    if (n_tokens < 1 || n_tokens > (1 << 30) || n_heads < 1 || n_heads > 65535 || head_dim < 1)
+        return REGENVC_ERR_BAD_SHAPE;
+    if (head_dim != kHeadDim || n_heads % kProjHeadsPerCta != 0) return REGENVC_ERR_UNSUPPORTED;
+    if (((uintptr_t)attn_out | (uintptr_t)w_o | (uintptr_t)y | (uintptr_t)b_o) & 15) return REGENVC_ERR_MISALIGNED;
+    const size_t C = (size_t)n_heads * kHeadDim;
+    const size_t ob = (size_t)n_tokens * C * 2, wb = C * C * 2;
+    if (overlaps(y, ob, attn_out, ob) || overlaps(y, ob, w_o, wb) || (b_o && overlaps(y, ob, b_o, C * 4)))
+        return REGENVC_ERR_ALIASING;
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev = 0;
+    DeviceState* st = nullptr;
+    int rc = device_state(&dev, &st);
+    if (rc != REGENVC_OK) return rc;
+    ProjParams pp{};
+    pp.bias = reinterpret_cast<const float*>(b_o);
+    pp.n_tokens = n_tokens;
+    pp.n_pad = (int)(((long long)n_tokens + kTile - 1) / kTile * kTile);
+    pp.C = (int)C;
+    pp.h = n_heads;
+    pp.grid = RopeGrid{nullptr, 1, 1, 1};
+    pp.status = st->status;
+    CUtensorMap tmap_o, tmap_w, tmap_y;
+    rc = make_tmap(&tmap_o, const_cast<void*>(attn_out), C, (uint64_t)n_tokens, C * 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
+    if (rc == REGENVC_OK)
+        rc = make_tmap(&tmap_w, const_cast<void*>(w_o), C, C, C * 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
+    if (rc == REGENVC_OK) rc = make_tmap(&tmap_y, y, C, (uint64_t)n_tokens, C * 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
+    if (rc != REGENVC_OK) return rc;
+    CUDA_TRY(launch_out_project(tmap_o, tmap_w, tmap_y, pp, st->sm_count, (cudaStream_t)stream));
+    launched();
+    return REGENVC_OK;
 }
 
 int regenvc_attn_forward_host(const void* q, const void* k, const void* v, void* out, int T, int H, int W, int n_heads,

@@ -96,6 +96,11 @@ cudaError_t configure_qkv_project();
 cudaError_t launch_qkv_project(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w, const CUtensorMap& tmap_q,
                                const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const ProjParams& p,
                                int sm_count, cudaStream_t stream);
+// Output projection y = o W_o^T + b_o (bf16 in, bf16 out) on pairs of CTAs (out_project_pair.cu); of ProjParams it
+// reads bias ([C] or nullptr), n_tokens, C, h and status.
+cudaError_t configure_out_project();
+cudaError_t launch_out_project(const CUtensorMap& tmap_o, const CUtensorMap& tmap_w, const CUtensorMap& tmap_y,
+                               const ProjParams& p, int sm_count, cudaStream_t stream);
 
 // Merge of token-major partial results of several key/value blocks.
 constexpr int kMaxMergeParts = 8;

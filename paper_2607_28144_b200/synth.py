@@ -24,6 +24,7 @@ ROPE_THETA = 10000.0
 
 # generator streams
 STREAM_Q, STREAM_K, STREAM_V, STREAM_CK, STREAM_CV, STREAM_SCALE, STREAM_X, STREAM_W, STREAM_B, STREAM_G = range(10)
+STREAM_WO, STREAM_BO = 10, 11
 
 
 @dataclass(frozen=True)
@@ -109,6 +110,15 @@ def block_inputs(w: Workload):
     b = 0.1 * torch.randn((3 * C,), generator=_gen(w.seed, STREAM_B), dtype=torch.float32)
     g = 0.5 + torch.rand((2, C), generator=_gen(w.seed, STREAM_G), dtype=torch.float32)
     return x, wq, b, g[0].contiguous(), g[1].contiguous(), 1e-6
+
+
+def out_proj_inputs(w: Workload):
+    """Inputs of the block's output projection: weights w_o [C, C] ~ N(0, 1/C) bf16 and bias [C] ~ N(0, 0.1^2) fp32
+    (stand-ins for trained weights, like block_inputs)."""
+    C = w.n_heads * w.head_dim
+    wo = (torch.randn((C, C), generator=_gen(w.seed, STREAM_WO), dtype=torch.float32) / C ** 0.5).to(torch.bfloat16)
+    bo = 0.1 * torch.randn((C,), generator=_gen(w.seed, STREAM_BO), dtype=torch.float32)
+    return wo, bo
 
 
 def bits(t: torch.Tensor) -> np.ndarray:
