@@ -146,8 +146,8 @@ int regenvc_attn_forward_prepared(const void* q_rot, const void* prepared, void*
  * heads of a token tile): otherwise REGENVC_ERR_UNSUPPORTED.  The thread blocks that share a token tile exchange
  * their partial sums of squares through 6 * T*H*W * n_heads bytes (plus counters) of the calling thread's
  * workspace -- regenvc_workspace_bytes(T*H*W, n_heads, 128) is always enough for a caller-supplied one -- and wait
- * for each other with the same bounded waits as everything else (REGENVC_ERR_TIMEOUT if the GPU is shared with
- * work that keeps part of the grid from becoming resident for half a second).  Asynchronous on `stream`; allocates
+ * for each other with the same bounded waits as everything else; the kernel is launched cooperatively (whole grid
+ * resident at once; REGENVC_ERR_CUDA if the device cannot grant that).  Asynchronous on `stream`; allocates
  * only the rotary table of a new (T, H, W, theta) and, the first time, the workspace.  Typical use:
  *     regenvc_qkv_rope_project(x, w, b, gq, gk, eps, q_rot, prepared, T, H, W, h, 128, theta, s);
  *     regenvc_attn_forward_prepared(q_rot, prepared, out, T*H*W, T*H*W, h, 128, s);

@@ -22,9 +22,9 @@
 // on the unit's counter; the epilogue warps (only they -- the producer and the MMA warp run ahead) wait until the
 // counter shows all slices and add the partial sums in slice order, so the result does not depend on timing.  The
 // wait is bounded like every other; it cannot deadlock because every CTA works through its slices in increasing
-// order and the whole grid is resident (grid <= number of SMs, one CTA per SM).  (A first form exchanged the sums
-// through distributed shared memory inside clusters of h/2 CTAs; clusters of 6 left 16 of this part's 148 SMs idle
-// and capped the head count at 16.)
+// order and the whole grid is resident (grid <= number of SMs, one CTA per SM, cooperative launch).  (A first form
+// exchanged the sums through distributed shared memory inside clusters of h/2 CTAs; clusters of 6 left 16 of this
+// part's 148 SMs idle and capped the head count at 16.)
 #include <cstddef>
 
 #include "common.cuh"
@@ -404,10 +404,21 @@ cudaError_t launch_qkv_project(const CUtensorMap& tmap_x, const CUtensorMap& tma
     // the counters of the units start at zero; the partial sums need no clearing (every slot is written before read)
     cudaError_t e = cudaMemsetAsync(p.unit_count, 0, (size_t)n_units * sizeof(int), stream);
     if (e != cudaSuccess) return e;
-    // one CTA per SM and never more CTAs than SMs: the whole grid is resident, which the waits between slices rely on
+    // One CTA per SM and never more CTAs than SMs, launched cooperatively: the waits between slices rely on the whole
+    // grid being resident at once, and a cooperative launch either guarantees that or fails (on a GPU whose SMs are
+    // partly taken it is refused instead of running into the bounded waits).
     const int grid = n_slices < sm_count ? n_slices : sm_count;
-    qkv_project_kernel<<<grid, kProjThreads, kProjSmem, stream>>>(tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kProjThreads);
+    cfg.dynamicSmemBytes = kProjSmem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, qkv_project_kernel, tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, p);
 }
 
 }  // namespace regenvc
