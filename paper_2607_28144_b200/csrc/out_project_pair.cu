@@ -13,10 +13,13 @@
 // c + n_clusters, ...
 //   warp 0      TMA producer of THIS CTA's operand halves; all bytes of a stage are counted on the leader's barrier
 //   warp 1      leader CTA: issues the pair MMAs (M = 256 over both CTAs, N = 256) and commits to the barriers of
-//               both CTAs.  Both CTAs: passes "my epilogue warps have read accumulator b" on to the leader.
-//   warps 2-9   epilogue of this CTA's 128 x 256 accumulator half: + bias, bf16, swizzled staging tile, tiled store
-// Two accumulators of 256 columns per CTA, used in turn.  Every TMA load here reads this GPU's own memory and
-// every CTA fetches its own tiles.
+//               both CTAs
+//   warps 2-9   epilogue of this CTA's 128 x 256 accumulator half: + bias, bf16, swizzled staging tile, tiled store;
+//               one of its threads tells the leader's barrier that this CTA has read accumulator b out
+// Two accumulators of 256 columns per CTA, used in turn.  (The hand-back of an accumulator first went through each
+// CTA's warp 1; a release-arrive at cluster scope from the thread that issues the MMAs waits for its earlier commits,
+// i.e. for the queued MMAs to finish, and left the tensor core idle for about 2 k cycles per slice.)  Every TMA load
+// here reads this GPU's own memory and every CTA fetches its own tiles.
 #include <cstddef>
 
 #include "common.cuh"
@@ -44,8 +47,8 @@ struct PairShared {
     uint64_t full[kStages];
     uint64_t empty[kStages];
     uint64_t acc_full[2];      // accumulator b holds a finished slice
-    uint64_t acc_read[2];      // this CTA's epilogue warps have read accumulator b out
-    uint64_t acc_empty[2];     // ... in BOTH CTAs (the leader's barrier; one arrival per CTA, from its warp 1)
+    uint64_t acc_empty[2];     // the epilogue warps of BOTH CTAs have read accumulator b out (the leader's barrier
+                               // counts; one arrival per CTA)
     uint32_t tmem_base;
     int abort_flag;
     alignas(16) float bias[kFeat];
@@ -148,7 +151,6 @@ out_project_pair_kernel(const __grid_constant__ CUtensorMap tmap_o, const __grid
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&sh->acc_full[b]), 1);
-            mbar_init(smem_u32(&sh->acc_read[b]), kEpiThreads);
             mbar_init(smem_u32(&sh->acc_empty[b]), 2);
         }
         sh->abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0) ? 1 : 0;
@@ -197,19 +199,13 @@ out_project_pair_kernel(const __grid_constant__ CUtensorMap tmap_o, const __grid
             for (int slice = slice0; ok && slice < n_slices; slice += slice_step, ++it) {
                 const int b = it & 1;
                 const uint32_t acc_tmem = tmem_base + b * kFeat;
+                if (rank != 0) break;      // only the leader issues MMAs
                 if (it >= 2) {
-                    // Accumulator b was last used two slices ago.  Each CTA's thread here waits until its own epilogue
-                    // warps have read it out and tells the leader; the leader goes on when both CTAs have said so.
-                    ok = mbar_wait(smem_u32(&sh->acc_read[b]), ((it >> 1) - 1) & 1, ctl);
-                    if (!ok) break;
-                    tc_fence_after();
-                    tc_fence_before();
-                    mbar_arrive_cluster(map_to_rank(smem_u32(&sh->acc_empty[b]), 0));
-                    if (rank == 0) ok = mbar_wait(smem_u32(&sh->acc_empty[b]), ((it >> 1) - 1) & 1, ctl);
+                    // accumulator b was last used two slices ago: both CTAs' epilogue warps must have read it out
+                    ok = mbar_wait(smem_u32(&sh->acc_empty[b]), ((it >> 1) - 1) & 1, ctl);
                     if (!ok) break;
                     tc_fence_after();
                 }
-                if (rank != 0) continue;   // only the leader issues MMAs
                 for (int kb = 0; kb < n_kb; ++kb, ++fill) {
                     const int s = fill % kStages;
                     ok = mbar_wait(smem_u32(&sh->full[s]), (fill / kStages) & 1, ctl);
@@ -273,11 +269,11 @@ out_project_pair_kernel(const __grid_constant__ CUtensorMap tmap_o, const __grid
                         *reinterpret_cast<uint4*>(my_stage + (col >> 6) * kOutBlockBytes + sw128_offset(row, (col >> 3) & 7)) = w;
                 }
             }
-            // this CTA's accumulator has been read out (warp 1 of this CTA passes that on to the leader)
             tc_fence_before();
-            mbar_arrive(smem_u32(&sh->acc_read[b]));
             fence_proxy_async_smem();
             epi_barrier();
+            // every epilogue thread of this CTA has its accumulator values: tell the leader
+            if (tid == 64) mbar_arrive_cluster(map_to_rank(smem_u32(&sh->acc_empty[b]), 0));
             if (tid == 64 && ok && tile_live) {
                 // rows past the last token fall outside the tensor map and are dropped by the store
 #pragma unroll

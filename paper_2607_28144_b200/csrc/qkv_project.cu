@@ -73,6 +73,15 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
     return v;
 }
 
+// Unit index -> (token tile, part: 0 q, 1 k, 2 v), part-major: all token tiles of q, then of k, then of v, so that
+// only one third of W_qkv is live at a time.  (With the three parts of a token tile next to each other the whole of
+// W_qkv is re-read every few token tiles; for 40 heads that is 157 MB, more than the L2 holds, and the kernel ran at
+// 0.94-0.99 PFLOP/s instead of 1.22.  x is read three times instead, from L2 or at a third of the weights' size.)
+struct Unit {
+    int tile, part;
+};
+__device__ __forceinline__ Unit decode_unit(int unit, int n_tiles) { return Unit{unit % n_tiles, unit / n_tiles}; }
+
 }  // namespace
 
 __global__ void __launch_bounds__(kProjThreads, 1)
@@ -88,8 +97,8 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_rank = p.h / kProjHeadsPerCta;               // slices per unit
     const int n_tiles = (p.n_tokens + kTile - 1) / kTile;
-    const int n_slices = 3 * n_tiles * n_rank;               // slice s: unit s / n_rank (token tile unit / 3, part unit % 3:
-    const int slice0 = blockIdx.x, slice_step = gridDim.x;   // 0 q, 1 k, 2 v), heads 2 (s % n_rank) and 2 (s % n_rank) + 1
+    const int n_slices = 3 * n_tiles * n_rank;               // slice s: unit s / n_rank (token tile and part: decode_unit),
+    const int slice0 = blockIdx.x, slice_step = gridDim.x;   // heads 2 (s % n_rank) and 2 (s % n_rank) + 1
     const int n_kb = p.C / kBK;
     const WaitCtl ctl{&sh->abort_flag, p.status, kStatusTimeout, kProjWaitNs};
     uint32_t tmem_base = 0;
@@ -125,8 +134,9 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             bool ok = true;
             for (int slice = slice0; ok && slice < n_slices; slice += slice_step) {
                 const int unit = slice / n_rank, pair = slice % n_rank;
-                const int n0 = (unit / 3) * kTile;
-                const int f0 = (unit % 3) * p.C + pair * kFeat;   // first row of W_qkv (output feature) of this slice
+                const Unit u = decode_unit(unit, n_tiles);
+                const int n0 = u.tile * kTile;
+                const int f0 = u.part * p.C + pair * kFeat;   // first row of W_qkv (output feature) of this slice
                 for (int kb = 0; kb < n_kb; ++kb, ++fill) {
                     const int s = fill % kProjStages, round = fill / kProjStages;
                     if (round > 0) ok = mbar_wait(smem_u32(&sh->empty[s]), (round - 1) & 1, ctl);
@@ -145,7 +155,7 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             int fill = 0, it = 0;
             bool ok = true;
             for (int slice = slice0; ok && slice < n_slices; slice += slice_step, ++it) {
-                const int part = (slice / n_rank) % 3, b = it & 1;
+                const int part = decode_unit(slice / n_rank, n_tiles).part, b = it & 1;
                 const uint32_t acc_tmem = tmem_base + b * kFeat;
                 // the accumulator must have been read out by the epilogue of the unit before last
                 if (it >= 2) ok = mbar_wait(smem_u32(&sh->acc_empty[b]), ((it >> 1) - 1) & 1, ctl);
@@ -185,7 +195,8 @@ qkv_project_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         int it = 0;
         for (int slice = slice0; slice < n_slices; slice += slice_step, ++it) {
             const int unit = slice / n_rank, pair = slice % n_rank;
-            const int part = unit % 3, n0 = (unit / 3) * kTile, b = it & 1;
+            const Unit u = decode_unit(unit, n_tiles);
+            const int part = u.part, n0 = u.tile * kTile, b = it & 1;
             const bool normed = part < 2;
             const uint32_t t_acc = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + b * kFeat + half * 128;
             // this unit's slice of the bias and of the norm gains (the previous unit's readers are past the barrier
