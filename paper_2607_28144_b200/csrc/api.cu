@@ -123,7 +123,7 @@ int device_state(int* dev_out, DeviceState** st_out) {
                 g_encode = (EncodeTiledFn)fn;
             }
             CUDA_TRY(configure_attn_pipelined());
-            CUDA_TRY(configure_qkv_project());
+            CUDA_TRY(configure_qkv_project_pair());
             CUDA_TRY(configure_out_project());
             CUDA_TRY(configure_attn_persistent());
             CUDA_TRY(cudaMalloc(&st.status, sizeof(int)));
@@ -204,10 +204,10 @@ int rope_table(DeviceState& st, int T, int H, int W, float theta, const float2**
 }
 
 int make_tmap(CUtensorMap* m, void* base, uint64_t inner, uint64_t outer, uint64_t row_bytes,
-              CUtensorMapDataType type = CU_TENSOR_MAP_DATA_TYPE_FLOAT16, uint32_t box_rows = 128) {
+              CUtensorMapDataType type = CU_TENSOR_MAP_DATA_TYPE_FLOAT16) {
     const cuuint64_t gdim[2] = {inner, outer};
     const cuuint64_t gstride[1] = {row_bytes};
-    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t box[2] = {64, 128};
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode(m, type, 2, base, gdim, gstride, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -618,8 +618,7 @@ int regenvc_qkv_rope_project(const void* x, const void* w_qkv, const void* b_qkv
         if (rc != REGENVC_OK) return rc;
     }
     ProjParams pp;
-    pp.unit_count = reinterpret_cast<int*>(ws);
-    pp.unit_sums = reinterpret_cast<float*>(ws + proj_count_bytes(n));
+    pp.unit_sums = reinterpret_cast<float*>(ws);
     pp.bias = reinterpret_cast<const float*>(b_qkv);
     pp.g_q = reinterpret_cast<const float*>(g_q);
     pp.g_k = reinterpret_cast<const float*>(g_k);
@@ -637,14 +636,13 @@ int regenvc_qkv_rope_project(const void* x, const void* w_qkv, const void* b_qkv
     CUtensorMap tmap_x, tmap_w, tmap_q, tmap_k, tmap_v;
     rc = make_tmap(&tmap_x, const_cast<void*>(x), C, (uint64_t)n, C * 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     if (rc == REGENVC_OK)
-        rc = make_tmap(&tmap_w, const_cast<void*>(w_qkv), C, 3 * C, C * 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
-                       kProjHeadsPerCta * kHeadDim);
+        rc = make_tmap(&tmap_w, const_cast<void*>(w_qkv), C, 3 * C, C * 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     if (rc == REGENVC_OK) rc = make_tmap(&tmap_q, q_rot, C, (uint64_t)n, C * 2);
     if (rc == REGENVC_OK) rc = make_tmap(&tmap_k, kp, kHeadDim, (uint64_t)n_heads * n_pad, kHeadDim * sizeof(__half));
     if (rc == REGENVC_OK)
         rc = make_tmap(&tmap_v, vt, (uint64_t)n_pad, (uint64_t)n_heads * kHeadDim, (uint64_t)n_pad * sizeof(__half));
     if (rc != REGENVC_OK) return rc;
-    CUDA_TRY(launch_qkv_project(tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, pp, st->sm_count, (cudaStream_t)stream));
+    CUDA_TRY(launch_qkv_project_pair(tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, pp, st->sm_count, (cudaStream_t)stream));
     launched();
     return own ? note_use(*own, (cudaStream_t)stream) : REGENVC_OK;
 }

@@ -68,8 +68,9 @@ struct AttnParams {
     float2* part_ml;          // [piece CTA][256 rows] (reference m in log2 units, row sum l)
 };
 
-// QKV projection with fused norm / rotation / operand-layout epilogue (producer of the attention operands).
-constexpr int kProjHeadsPerCta = 2;   // a CTA computes 128 tokens x two heads of one of q, k, v per work unit
+// QKV projection with fused norm / rotation / operand-layout epilogue (producer of the attention operands), on pairs
+// of CTAs (qkv_project_pair.cu).
+constexpr int kProjHeadsPerCta = 2;   // a slice of the projection kernels is 256 output features = two heads
 struct ProjParams {
     const float* bias;        // [3C] or nullptr
     const float* g_q;         // [C] RMS-norm gains of q (nullptr: ones)
@@ -78,24 +79,19 @@ struct ProjParams {
     int n_tokens, n_pad, C, h;
     RopeGrid grid;
     int* status;
-    // scratch of the norm's sum over all features: per (128-token tile, q/k/v) unit one counter of the slices that
-    // have published their partial row sums, and the sums themselves [unit][slice][128 tokens]
-    int* unit_count;
+    // scratch of the norm's sum over all features: the partial row sums of every (128-token tile, q/k/v) unit and
+    // slice, [unit][slice][128 tokens]; a slot that still holds the all-ones pattern has not been written yet
     float* unit_sums;
 };
-// Bytes of that scratch for n_tokens tokens and h heads (counters first, 256-byte aligned, then the sums).
-inline size_t proj_count_bytes(long long n_tokens) {
-    const size_t n_units = 3 * (size_t)((n_tokens + kTile - 1) / kTile);
-    return (n_units * sizeof(int) + 255) / 256 * 256;
-}
+// Bytes of that scratch for n_tokens tokens and h heads.
 inline size_t proj_scratch_bytes(long long n_tokens, int h) {
     const size_t n_units = 3 * (size_t)((n_tokens + kTile - 1) / kTile);
-    return proj_count_bytes(n_tokens) + n_units * (size_t)(h / kProjHeadsPerCta) * kTile * sizeof(float);
+    return n_units * (size_t)(h / kProjHeadsPerCta) * kTile * sizeof(float);
 }
-cudaError_t configure_qkv_project();
-cudaError_t launch_qkv_project(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w, const CUtensorMap& tmap_q,
-                               const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const ProjParams& p,
-                               int sm_count, cudaStream_t stream);
+cudaError_t configure_qkv_project_pair();
+cudaError_t launch_qkv_project_pair(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w, const CUtensorMap& tmap_q,
+                                    const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const ProjParams& p,
+                                    int sm_count, cudaStream_t stream);
 // Output projection y = o W_o^T + b_o (bf16 in, bf16 out) on pairs of CTAs (out_project_pair.cu); of ProjParams it
 // reads bias ([C] or nullptr), n_tokens, C, h and status.
 cudaError_t configure_out_project();
