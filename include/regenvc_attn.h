@@ -144,10 +144,11 @@ int regenvc_attn_forward_prepared(const void* q_rot, const void* prepared, void*
  * Arithmetic: bf16 products accumulated in fp32, norm and rotation in fp32, one rounding to fp16.  A result
  * beyond the fp16 range sets the sticky REGENVC_ERR_RANGE status.  n_heads must be even (a thread block computes two
  * heads of a token tile): otherwise REGENVC_ERR_UNSUPPORTED.  The thread blocks that share a token tile exchange
- * their partial sums of squares through 6 * T*H*W * n_heads bytes (plus counters) of the calling thread's
- * workspace -- regenvc_workspace_bytes(T*H*W, n_heads, 128) is always enough for a caller-supplied one -- and wait
- * for each other with the same bounded waits as everything else; the kernel is launched cooperatively (whole grid
- * resident at once; REGENVC_ERR_CUDA if the device cannot grant that).  Asynchronous on `stream`; allocates
+ * their partial sums of squares through 6 * n_pad * n_heads bytes (n_pad = T*H*W rounded up to 128) of the calling
+ * thread's workspace -- regenvc_workspace_bytes(T*H*W, n_heads, 128) is always enough for a caller-supplied one --
+ * and wait for each other with the same bounded waits as everything else (the grid never exceeds what the device
+ * holds at once; REGENVC_ERR_TIMEOUT if the GPU is shared with work that keeps part of it from becoming resident for
+ * half a second).  Asynchronous on `stream`; allocates
  * only the rotary table of a new (T, H, W, theta) and, the first time, the workspace.  Typical use:
  *     regenvc_qkv_rope_project(x, w, b, gq, gk, eps, q_rot, prepared, T, H, W, h, 128, theta, s);
  *     regenvc_attn_forward_prepared(q_rot, prepared, out, T*H*W, T*H*W, h, 128, s);

@@ -25,7 +25,7 @@
 // counts itself in on the (token tile, part) counter; the epilogue warps (only they) wait until the counter shows all
 // slices and add the partial sums in slice order, so the result does not depend on timing.  The wait is bounded like
 // every other; it cannot deadlock because every cluster works through its slices in increasing order and the whole
-// grid is resident (grid <= number of SMs, one CTA per SM).
+// grid is resident (never more pairs than the device holds at once, one CTA per SM).
 // An accumulator is handed back to the leader's MMA thread by ONE epilogue thread per CTA (cluster-scope arrive on the
 // leader's barrier) -- not by the MMA-issuing thread itself, whose release-arrive would wait for its queued MMAs.
 #include <cstddef>
@@ -452,20 +452,20 @@ cudaError_t launch_qkv_project_pair(const CUtensorMap& tmap_x, const CUtensorMap
     cudaError_t e = cudaMemsetAsync(p.unit_sums, 0xff, (size_t)3 * n_tiles * (p.h / kProjHeadsPerCta) * kTile * sizeof(float),
                                     stream);
     if (e != cudaSuccess) return e;
-    // Pairs of CTAs, one CTA per SM and never more CTAs than SMs, launched cooperatively: the waits between slices rely
-    // on the whole grid being resident at once, and a cooperative launch either guarantees that or fails.
+    // Pairs of CTAs, one CTA per SM, and never more pairs than the device holds at once: the waits between slices rely
+    // on the whole grid being resident.  (The cooperative launch attribute, which would have the driver guarantee
+    // that, was tried: with it this kernel fails to launch under the profiler.  On a device shared with other work
+    // part of the grid may stay out; the waits then run out and the sticky status reports it.)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * (unsigned)(sm_count / 2));
     cfg.blockDim = dim3(kProjThreads);
     cfg.dynamicSmemBytes = kProjSmem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeCooperative;
-    attr[1].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     // how many pairs the device can hold at once (fewer than SMs / 2 where a GPC has an odd number of free SMs)
@@ -475,7 +475,6 @@ cudaError_t launch_qkv_project_pair(const CUtensorMap& tmap_x, const CUtensorMap
     const int pairs = n_slices < resident ? n_slices : resident;
     if (pairs < 1) return cudaErrorInvalidConfiguration;
     cfg.gridDim = dim3(2 * (unsigned)pairs);
-    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, qkv_project_pair_kernel, tmap_x, tmap_w, tmap_q, tmap_k, tmap_v, p);
 }
 
