@@ -1,5 +1,5 @@
-// Thin inline-PTX wrappers for sm_100a: mbarrier, TMA (bulk tensor copies, no
-// multicast), tcgen05 (tensor-memory allocation, UMMA issue/commit, TMEM
+// Thin inline-PTX wrappers for sm_100a: mbarrier, TMA (bulk tensor copies, every CTA
+// loading its own tiles), tcgen05 (tensor-memory allocation, UMMA issue/commit, TMEM
 // load/store) and the fences that order them.  Every spin on an mbarrier is
 // bounded: on expiry the waiter records a sticky status and raises a CTA-wide
 // abort flag, after which all further waits fall through so that the CTA can
