@@ -278,7 +278,8 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
         int visit = 0;  // key tiles done so far over all items = completed phases of s_full, p_full, o_full (both tiles)
 
         for (int item = first_item; item < n_items; item += item_step) {
-            const int n_active = decode_item(item, p).n_active;
+            const PItem wi = decode_item(item, p);   // kept for the stores at the end: the divisions stay off that path
+            const int n_active = wi.n_active;
             if (n_active == 0) continue;
             float m_ref[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
 
@@ -426,7 +427,6 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
                     fence_proxy_async_smem();
                     softmax_barrier();
                     if (tid == 0 && ok) {
-                        const PItem wi = decode_item(item, p);
                         const uint32_t src = smem_u32(sOut);
                         tma_store_2d(&tmap_out, wi.head * kHeadDim, wi.q0 + t * kTile, src);
                         tma_store_2d(&tmap_out, wi.head * kHeadDim + 64, wi.q0 + t * kTile, src + kBlockBytes);
