@@ -73,7 +73,21 @@ __device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
 __device__ __forceinline__ void softmax_barrier() {
     asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");
 }
-// The same barrier with an OR-reduction of one predicate per thread: every thread of the row group learns
+// Barrier 1 with an OR-reduction of one predicate per thread: every softmax thread learns whether any of them
+// raised the flag.
+__device__ __forceinline__ bool softmax_any(bool flag) {
+    uint32_t any;
+    asm volatile(
+        "{\n\t.reg .pred pin, pout;\n\t"
+        "setp.ne.u32 pin, %1, 0;\n\t"
+        "bar.red.or.pred pout, 1, %2, pin;\n\t"
+        "selp.u32 %0, 1, 0, pout;\n\t}"
+        : "=r"(any)
+        : "r"(static_cast<uint32_t>(flag)), "n"(kSoftmaxThreads)
+        : "memory");
+    return any != 0;
+}
+// A row group's barrier with an OR-reduction of one predicate per thread: every thread of the row group learns
 // whether any of them raised the flag, without touching shared memory.
 __device__ __forceinline__ bool row_group_any(int g, bool flag) {
     uint32_t any;

@@ -20,11 +20,19 @@
 // Softmax keeps, per row, a reference m (log2 domain) and a row sum l.  m is set from the first tile's row
 // maximum and afterwards only raised when a probability would leave the fp16 range (p = 2^(s - m) > 65504),
 // so the probabilities of a tile are formed directly against the reference of the earlier tiles as soon as
-// the scores arrive; one named barrier with an OR-reduction per tile lets the warps that share 32 rows agree
-// that nothing saturated, and the rescale of the O accumulator (with a redo of the tile) is rare.
+// the scores arrive.  A saturated probability shows in the fp32 sum of its thread's part of the row.
+// The CTA first runs its key tiles OPTIMISTICALLY: every thread only remembers whether any of its sums
+// saturated, nothing is exchanged per tile (the per-tile agreement of the four warps that share 32 rows cost
+// 3.6 % of the kernel although it practically never fires), and at the end of the item one OR-reduction over
+// the softmax warps says whether the pass was clean.  If it was not, the result of the pass is discarded and
+// the whole item is run again CAREFULLY: one named barrier with an OR-reduction per tile lets the warps of a
+// row group agree on a saturation at once, the row maximum is taken, the reference raised, O rescaled and the
+// tile redone.  The control warps learn the verdict through an mbarrier and stream the tiles a second time.
 #include "common.cuh"
 #include "attn_core.cuh"
 #include "rope.cuh"
+
+#include <type_traits>
 
 namespace regenvc {
 
@@ -41,8 +49,10 @@ struct Barriers {
     uint64_t s_full[2];
     uint64_t p_full[2];
     uint64_t o_full[2];
+    uint64_t verdict;        // the softmax warps have judged the optimistic pass (second_pass is valid)
     uint32_t tmem_base;
     int abort_flag;
+    int second_pass;         // 1: a probability saturated in the optimistic pass, the item is run again
 };
 static_assert(sizeof(Barriers) <= 256, "barrier block too large");
 
@@ -96,6 +106,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             mbar_init(smem_u32(&bar->p_full[t]), kSoftmaxThreads);
             mbar_init(smem_u32(&bar->o_full[t]), 1);
         }
+        mbar_init(smem_u32(&bar->verdict), 1);
         // a sticky error from an earlier kernel makes this CTA skip its work (every bounded wait falls through)
         bar->abort_flag = (*reinterpret_cast<volatile int*>(p.status) != 0) ? 1 : 0;
         fence_mbar_init();
@@ -131,19 +142,28 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 }
             }
             const int total = 2 * n_tiles;
-            for (int i = 0; i < total; ++i) {
-                const int slot = i % kStages, round = i / kStages;
-                if (round > 0 && !mbar_wait(smem_u32(&bar->kv_empty[slot]), (round - 1) & 1, ctl)) break;
-                const uint32_t full = smem_u32(&bar->kv_full[slot]);
-                const uint32_t dst = smem_u32(sKV + slot * kTileBytes);
-                const int kv0 = (kv_tile0 + (i >> 1)) * kTile;
-                mbar_expect_tx(full, kTileBytes);
-                if ((i & 1) == 0) {
-                    tma_load_2d(dst, &tmap_k, 0, head * p.n_kv_pad + kv0, full);
-                    tma_load_2d(dst + kBlockBytes, &tmap_k, 64, head * p.n_kv_pad + kv0, full);
-                } else {
-                    tma_load_2d(dst, &tmap_v, kv0, head * kHeadDim, full);
-                    tma_load_2d(dst + kBlockBytes, &tmap_v, kv0 + 64, head * kHeadDim, full);
+            bool ok = true;
+            for (int pass = 0; ok && pass < 2; ++pass) {   // the ring index runs on through the second pass
+                for (int i = 0; ok && i < total; ++i) {
+                    const int g = pass * total + i;
+                    const int slot = g % kStages, round = g / kStages;
+                    if (round > 0) ok = mbar_wait(smem_u32(&bar->kv_empty[slot]), (round - 1) & 1, ctl);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&bar->kv_full[slot]);
+                    const uint32_t dst = smem_u32(sKV + slot * kTileBytes);
+                    const int kv0 = (kv_tile0 + (i >> 1)) * kTile;
+                    mbar_expect_tx(full, kTileBytes);
+                    if ((i & 1) == 0) {
+                        tma_load_2d(dst, &tmap_k, 0, head * p.n_kv_pad + kv0, full);
+                        tma_load_2d(dst + kBlockBytes, &tmap_k, 64, head * p.n_kv_pad + kv0, full);
+                    } else {
+                        tma_load_2d(dst, &tmap_v, kv0, head * kHeadDim, full);
+                        tma_load_2d(dst + kBlockBytes, &tmap_v, kv0 + 64, head * kHeadDim, full);
+                    }
+                }
+                if (pass == 0 && ok) {
+                    ok = mbar_wait(smem_u32(&bar->verdict), 0, ctl);
+                    if (!ok || !*reinterpret_cast<volatile int*>(&bar->second_pass)) break;
                 }
             }
         }
@@ -155,35 +175,45 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
             const uint32_t idesc_qk = p.qk_bf16 ? kIdescBf16 : kIdesc;
             bool ok = mbar_wait(smem_u32(&bar->q_full[0]), 0, ctl);
             if (ok && tile1_active) ok = mbar_wait(smem_u32(&bar->q_full[1]), 0, ctl);
-            if (ok) ok = mbar_wait(smem_u32(&bar->kv_full[0]), 0, ctl);
-            if (ok) {
+            // pass 0: the optimistic run; pass 1 (only after a saturation): the same tiles again.  Ring index and
+            // visit count (the phases of s_full / p_full / o_full) run on through the second pass.
+            for (int pass = 0; ok && pass < 2; ++pass) {
+                const int g0 = pass * 2 * n_tiles, v0 = pass * n_tiles;
+                ok = mbar_wait(smem_u32(&bar->kv_full[g0 % kStages]), (g0 / kStages) & 1, ctl);
+                if (!ok) break;
                 tc_fence_after();
+                // (on the second pass the score columns are free: the last P.V of the first pass, issued earlier by
+                // this thread, reads them before these MMAs run)
                 for (int t = 0; t < n_active; ++t) {
-                    issue_qk(tmem_base + t * 128, t ? sQ1 : sQ0, smem_u32(sKV), idesc_qk);
+                    issue_qk(tmem_base + t * 128, t ? sQ1 : sQ0, smem_u32(sKV + (g0 % kStages) * kTileBytes), idesc_qk);
                     umma_commit(smem_u32(&bar->s_full[t]));
                 }
-                umma_commit(smem_u32(&bar->kv_empty[0]));
-            }
-            for (int j = 0; ok && j < n_tiles; ++j) {
-                const int iv = 2 * j + 1, ik = 2 * j + 2;
-                const int slot_v = iv % kStages, slot_k = ik % kStages;
-                const bool more = j + 1 < n_tiles;
-                ok = mbar_wait(smem_u32(&bar->kv_full[slot_v]), (iv / kStages) & 1, ctl);
-                if (ok && more) ok = mbar_wait(smem_u32(&bar->kv_full[slot_k]), (ik / kStages) & 1, ctl);
-                for (int t = 0; ok && t < n_active; ++t) {
-                    ok = mbar_wait(smem_u32(&bar->p_full[t]), j & 1, ctl);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_pv(tmem_base + 256 + t * 128, tmem_base + t * 128, smem_u32(sKV + slot_v * kTileBytes), j > 0);
-                    umma_commit(smem_u32(&bar->o_full[t]));
-                    if (more) {
-                        issue_qk(tmem_base + t * 128, t ? sQ1 : sQ0, smem_u32(sKV + slot_k * kTileBytes), idesc_qk);
-                        umma_commit(smem_u32(&bar->s_full[t]));
+                umma_commit(smem_u32(&bar->kv_empty[g0 % kStages]));
+                for (int j = 0; ok && j < n_tiles; ++j) {
+                    const int iv = g0 + 2 * j + 1, ik = g0 + 2 * j + 2;
+                    const int slot_v = iv % kStages, slot_k = ik % kStages;
+                    const bool more = j + 1 < n_tiles;
+                    ok = mbar_wait(smem_u32(&bar->kv_full[slot_v]), (iv / kStages) & 1, ctl);
+                    if (ok && more) ok = mbar_wait(smem_u32(&bar->kv_full[slot_k]), (ik / kStages) & 1, ctl);
+                    for (int t = 0; ok && t < n_active; ++t) {
+                        ok = mbar_wait(smem_u32(&bar->p_full[t]), (v0 + j) & 1, ctl);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(tmem_base + 256 + t * 128, tmem_base + t * 128, smem_u32(sKV + slot_v * kTileBytes), j > 0);
+                        umma_commit(smem_u32(&bar->o_full[t]));
+                        if (more) {
+                            issue_qk(tmem_base + t * 128, t ? sQ1 : sQ0, smem_u32(sKV + slot_k * kTileBytes), idesc_qk);
+                            umma_commit(smem_u32(&bar->s_full[t]));
+                        }
+                    }
+                    if (ok) {
+                        umma_commit(smem_u32(&bar->kv_empty[slot_v]));
+                        if (more) umma_commit(smem_u32(&bar->kv_empty[slot_k]));
                     }
                 }
-                if (ok) {
-                    umma_commit(smem_u32(&bar->kv_empty[slot_v]));
-                    if (more) umma_commit(smem_u32(&bar->kv_empty[slot_k]));
+                if (pass == 0 && ok) {
+                    ok = mbar_wait(smem_u32(&bar->verdict), 0, ctl);
+                    if (!ok || !*reinterpret_cast<volatile int*>(&bar->second_pass)) break;
                 }
             }
         }
@@ -208,27 +238,36 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
         const float scale = p.scale_log2;
         const uint64_t scale2 = pack2(scale, scale);
         const uint32_t opaque_zero = static_cast<uint32_t>(p.n_kv) >> 31;  // 0, but not to the compiler
-        float m_ref[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+        float m_ref[2], l_run[2];
         bool ok = true;  // false once a wait expired: keep the loop structure (named barriers) but skip the work
+        bool sat = false;  // optimistic pass: one of this thread's partial row sums saturated
         // the one key tile of the sequence that is partly padding (if this CTA has it), and how many of this
         // thread's columns of that tile are real keys
         const int j_ragged = (p.n_kv % kTile != 0 && kv_tile0 + n_tiles == n_tiles_total) ? n_tiles - 1 : -1;
         const int valid_last = p.n_kv - (n_tiles_total - 1) * kTile - part * kColsPerThread;
 
-        for (int j = 0; j < n_tiles; ++j) {
+        // One pass over the CTA's key tiles.  kCareful = false: optimistic (see the header), saturation is only
+        // recorded in `sat`; true: the warps of a row group agree per tile and redo a saturated tile against a higher
+        // reference.  v0: visits done before this pass (the phases of s_full / p_full / o_full run on).
+        auto run_pass = [&](auto careful_tag, const int v0) {
+          constexpr bool kCareful = decltype(careful_tag)::value;
+          m_ref[0] = m_ref[1] = -INFINITY;
+          l_run[0] = l_run[1] = 0.f;
+          for (int j = 0; j < n_tiles; ++j) {
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
                 if (t >= n_active) continue;
                 const uint32_t t_S = lane_base + t * 128 + part * kColsPerThread;
                 const uint32_t t_O = lane_base + 256 + t * 128 + part * kColsPerThread;
-                if (ok) ok = mbar_wait(smem_u32(&bar->s_full[t]), j & 1, ctl);
+                if (ok) ok = mbar_wait(smem_u32(&bar->s_full[t]), (v0 + j) & 1, ctl);
                 ok = __all_sync(0xffffffffu, ok);  // keep the warp-wide TMEM instructions below convergent
                 tc_fence_after();
                 // From the second tile on, the probabilities of each 32-column chunk are formed as soon as it
                 // arrives, against the reference m_ref of the earlier tiles; no maximum is taken.  Probabilities
                 // saturate at 65504 when rounded to fp16, and a saturated one makes the fp32 sum of its part reach
-                // 65504, which the threads of the row detect by exchanging their sums; only then (and on the first
-                // tile) the row maximum is taken, the reference raised, O rescaled and the tile redone.
+                // 65504.  Optimistic pass: the thread remembers it.  Careful pass: the threads of the row group agree
+                // on it; only then (and on the first tile of either pass) the row maximum is taken, the reference
+                // raised, O rescaled and the tile redone.
                 uint32_t sr[kColsPerThread];
                 uint64_t negm2 = pack2(-m_ref[t], -m_ref[t]);
                 uint64_t sum_a = 0, sum_b = 0;  // packed partial row sums
@@ -257,9 +296,15 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     unpack2(add2(sum_a, sum_b), s0, s1);
                     part_sum = s0 + s1;
                 }
-                // One barrier with an OR-reduction tells the threads sharing these 32 rows whether any part of any
-                // row saturated (or this is the first tile); only then do they exchange anything.
-                const bool any_redo = row_group_any(warp & 3, !stream || !(part_sum < 65504.0f));
+                // Careful pass: one barrier with an OR-reduction tells the threads sharing these 32 rows whether any
+                // part of any row saturated (or this is the first tile); only then do they exchange anything.
+                bool any_redo;
+                if (kCareful) {
+                    any_redo = row_group_any(warp & 3, !stream || !(part_sum < 65504.0f));
+                } else {
+                    any_redo = !stream;                               // uniform over the CTA
+                    if (stream) sat |= !(part_sum < 65504.0f);
+                }
                 if (any_redo) {
                     // Rare after the first tile.  All threads of the row group take this branch together: row
                     // maximum, a higher reference for the rows whose maximum exceeds theirs, rescale of this
@@ -282,7 +327,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                     const float m_tile = mx_row * scale;
                     const bool raise = m_tile > m_ref[t];  // always on the first tile (reference starts at -inf)
                     if (j > 0) {
-                        if (ok) ok = mbar_wait(smem_u32(&bar->o_full[t]), (j - 1) & 1, ctl);
+                        if (ok) ok = mbar_wait(smem_u32(&bar->o_full[t]), (v0 + j - 1) & 1, ctl);
                         ok = __all_sync(0xffffffffu, ok);
                         tc_fence_after();
                         const float alpha = raise ? ex2_approx(m_ref[t] - m_tile) : 1.0f;
@@ -319,7 +364,17 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bar->p_full[t]));
             }
+          }
+        };
+        run_pass(std::false_type{}, 0);
+        // verdict on the optimistic pass, for these warps and (through the mbarrier) for the control warps
+        const bool again = softmax_any(sat);
+        if (tid == 0) {
+            bar->second_pass = again ? 1 : 0;
+            mbar_arrive(smem_u32(&bar->verdict));
         }
+        if (again) run_pass(std::true_type{}, n_tiles);
+        const int v_last = (again ? 2 : 1) * n_tiles - 1;   // the visit whose P.V the epilogue waits for
 
         // epilogue: O / l -> bf16 -> out; each thread owns kColsPerThread of the 128 output columns of its row
         for (int t = 0; t < n_active; ++t) {
@@ -329,7 +384,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
 #pragma unroll
             for (int o = 0; o < kSplit; ++o) l_row += xch->l[t][row][o];
             const float inv_l = 1.0f / l_row;
-            if (ok) ok = mbar_wait(smem_u32(&bar->o_full[t]), (n_tiles - 1) & 1, ctl);
+            if (ok) ok = mbar_wait(smem_u32(&bar->o_full[t]), v_last & 1, ctl);
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
             const uint32_t t_O = lane_base + 256 + t * 128 + part * kColsPerThread;
