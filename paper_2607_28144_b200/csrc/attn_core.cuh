@@ -46,16 +46,23 @@ struct RowExchange {
     float l[2][kTile][kSplit];     // row sums at the end: [tile][row][part]
 };
 
+// sign(x) * min(|x|, bound), bound > 0: the clamp to [-bound, bound] in one instruction.
+__device__ __forceinline__ float clamp_sym(float x, float bound) {
+    float y;
+    asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(y) : "f"(x), "f"(bound));
+    return y;
+}
+
 // 2^x for a packed pair on the FMA/ALU pipes: x = n + f with n = round(x), f in [-0.5, 0.5];
 // 2^f by a degree-3 minimax polynomial (max relative error 7.5e-5, below fp16 rounding of P),
-// 2^n by adding n to the exponent field.  x is clamped to [-125, 126] so that the exponent cannot wrap at
-// either end: a score far above the reference then still gives a probability of about 2^126, which saturates
+// 2^n by adding n to the exponent field.  x is clamped to [-125, 125] so that the exponent cannot wrap at
+// either end: a score far above the reference then still gives a probability of about 2^125, which saturates
 // the fp16 conversion, pushes the part's row sum past 65504 and so requests the raise of the reference, exactly
 // as the infinity of the MUFU path does.
 __device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
     float x0, x1;
     unpack2(x2, x0, x1);
-    x2 = pack2(fminf(fmaxf(x0, -125.0f), 126.0f), fminf(fmaxf(x1, -125.0f), 126.0f));
+    x2 = pack2(clamp_sym(x0, 125.0f), clamp_sym(x1, 125.0f));
     const float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
     const uint64_t r2 = add2(x2, pack2(kMagic, kMagic));
     const uint64_t n2 = add2(r2, pack2(-kMagic, -kMagic));
