@@ -214,6 +214,27 @@ def test_one_key_far_above_the_reference_of_the_earlier_tiles(key, amp):
     assert_parity(gpu, ref, float(v.float().abs().max()), f"jump at key {key}, amplitude {amp}")
 
 
+@pytest.mark.parametrize("key", [900, 1290])
+def test_a_saturation_in_one_work_item_only(key):
+    """Eleven key tiles (the one-CTA-per-item kernel, not the persistent one), five work items per head.  The query
+    rows 300..329 of head 0 and ONE late key point the same way with a score about 200 log2 units above everything
+    else: the optimistic pass saturates in that work item alone, which is run again carefully (reference raised,
+    accumulator rescaled) while every other item keeps the result of its clean first pass.  Those rows must equal
+    the key's value vector, all others ordinary attention."""
+    n_q, n_kv, h = 1100, 1300, 2
+    rng = np.random.default_rng(43)
+    q = rng.standard_normal((n_q, h, D)).astype(np.float32)
+    k = rng.standard_normal((n_kv, h, D)).astype(np.float32)
+    q[300:330, 0] = 3.5
+    k[key, 0] = 3.5
+    q, k, v = synth.from_f32(q), synth.from_f32(k), _rand(rng, n_kv, h)
+    gpu = f64(run_gpu_cross(q, k, v))
+    ref = oracle.cross_attention(synth.bits(q), synth.bits(k), synth.bits(v))
+    np.testing.assert_allclose(ref[300:330, 0], np.broadcast_to(f64(v)[key, 0], (30, D)), atol=1e-9)
+    assert_parity(gpu, ref, float(v.float().abs().max()), f"one saturating work item, key {key}")
+    assert_parity(gpu[300:330, :1], ref[300:330, :1], float(v.float().abs().max()), "the saturated rows")
+
+
 def test_heads_are_independent_on_the_gpu():
     T, H, W, h = 2, 9, 10, 4
     N = T * H * W
