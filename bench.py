@@ -93,7 +93,7 @@ class ClockSampler:
                 self.power.append(self.nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
             except Exception:
                 pass
-            time.sleep(0.005)
+            time.sleep(0.001)
 
     def start(self):
         if self.nv is not None:
