@@ -9,8 +9,8 @@
 //     accumulator columns are handed back through o_free when the softmax warps have loaded them);
 //   * barriers, tensor memory and the tensor maps are set up once per CTA.
 // Roles, tensor-memory map and the UMMA sequences are those of attn_pipelined.cu; the softmax is that kernel's careful
-// form (the warps of a row group agree on a saturation tile by tile: with four key tiles per item a second pass over
-// the item would cost more than the four barriers).  Shared memory:
+// form (the warps of a row group agree on a saturation tile by tile; there is no optimistic pass here, because by the
+// time an item's verdict would be known the control warps are already streaming the next item).  Shared memory:
 // Q0, Q1, a 4-slot K'/V't ring and one 32 KB staging tile for the output (the query buffers cannot double as
 // staging here because the next item's tiles arrive while the epilogue runs; writing the output rows straight
 // from registers, 16 bytes per thread and store, was measured 13 us slower per call at the 480x832 window).
