@@ -3,8 +3,6 @@
 #pragma once
 #include <cstdint>
 
-#include "ptx.cuh"
-
 namespace regenvc {
 
 namespace {
@@ -12,9 +10,6 @@ namespace {
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// The two halves of that barrier, for warps that have nothing to publish and can do other work in between.
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t n;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(n));
@@ -75,46 +70,6 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 // accesses at cluster scope.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-// Arrival on a barrier of either CTA of the pair (shared::cluster address) without cluster-scope ordering of
-// ordinary memory: for hand-overs whose payload lives in tensor memory (made visible by tcgen05.wait / fence) or
-// is only the fact of the arrival itself.  The cluster-scope release of mbar_arrive_cluster costs hundreds of cycles.
-__device__ __forceinline__ void mbar_arrive_peer(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-// One 32-bit word into the shared memory of either CTA of the pair (shared::cluster address).
-__device__ __forceinline__ void st_shared_peer(uint32_t addr, uint32_t v) {
-    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
-// Bounded wait on a barrier of THIS CTA whose arrivals come from both CTAs of the pair with cluster-scope release
-// (mbar_arrive_cluster) and guard ordinary shared-memory words written from the other CTA: acquire at cluster scope.
-__device__ __forceinline__ bool mbar_wait_acq_cluster(uint32_t bar, uint32_t parity, const WaitCtl& ctl) {
-    uint64_t t0 = 0;
-    uint32_t spins = 0;
-    while (true) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (done) return true;
-        if ((++spins & 255u) == 0) {
-            if (*ctl.abort_flag) return false;
-            const uint64_t now = global_timer_ns();
-            if (t0 == 0) {
-                t0 = now;
-            } else if (now - t0 > ctl.limit_ns) {
-                *ctl.abort_flag = 1;
-                atomicCAS(ctl.status, 0, ctl.code);
-                return false;
-            }
-        }
-    }
 }
 
 }  // namespace
