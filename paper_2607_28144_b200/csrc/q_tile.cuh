@@ -31,6 +31,10 @@ __device__ __forceinline__ void load_rotate_q_tiles(const AttnParams& p, int hea
             if (n < p.n_q)
                 raw[t][it] = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)n * p.h + head) * kHeadDim) + chunk);
         }
+    // Grid position of this thread's first row by division, of its later rows (kRowsPerPass tokens further each) by
+    // stepping: the two integer divisions per row were the largest part of this routine's instructions.
+    TokenPos pos = {0, 0, 0};
+    if (p.rope) pos = token_pos(q0 + (tid >> 4) + p.q_pos_offset, p.grid);
 #pragma unroll
     for (int t = 0; t < kTilesQ; ++t)
 #pragma unroll
@@ -39,7 +43,17 @@ __device__ __forceinline__ void load_rotate_q_tiles(const AttnParams& p, int hea
             const int n = q0 + t * kTile + row;
             float x[8];
             bf16x8_to_float(raw[t][it], x);
-            if (p.rope && n < p.n_q) rope_rotate8(x, p.grid, token_pos(n + p.q_pos_offset, p.grid), rc);
+            if (p.rope) {
+                if (n < p.n_q) rope_rotate8(x, p.grid, pos, rc);
+                pos.x += kRowsPerPass;   // the next row of this thread
+                while (pos.x >= p.grid.W) {
+                    pos.x -= p.grid.W;
+                    if (++pos.y == p.grid.H) {
+                        pos.y = 0;
+                        ++pos.t;
+                    }
+                }
+            }
             uint4 packed;
             packed.x = pack_f16x2(x[0], x[1]);
             packed.y = pack_f16x2(x[2], x[3]);
