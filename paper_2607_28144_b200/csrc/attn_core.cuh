@@ -126,14 +126,13 @@ __device__ __forceinline__ void row_group_barrier(int g) {
 // packed fp32 pairs; pair c of every eight uses the polynomial when bit (c % 8) of kMask is set, the MUFU
 // otherwise, which splits the exponentials between the two pipes.  The fp32 probabilities are also added
 // into two packed partial row sums.
-// kExpGroup < 16 works the 16 pairs off in groups: every later group's FMAs are made to depend on the group before's
-// last conversion (through `zero`, a value that is 0 but that the compiler cannot know), which keeps the compiler
-// from gathering all FMAs, then all MUFU operations, then all additions and conversions of the chunk into three
-// long phases.  With the per-tile agreement barrier in the loop, groups of eight were 1.2 % faster than none (the four
-// warps of a scheduler ran the code in step and met on the same pipe less often); since the barrier left the common
-// path the ungrouped form is the faster one by about 1 % (isolated launches and under the power cap), so 16 it is.
+// The 16 pairs are worked off as two groups of eight: the second group's FMAs are made to depend on the first
+// group's last conversion (through `zero`, a value that is 0 but that the compiler cannot know), which keeps the
+// compiler from gathering all FMAs, then all MUFU operations, then all additions and conversions of the chunk
+// into three long phases; the warps of a scheduler then meet on the same pipe less often.  Measured on the shipped
+// kernel: groups of eight 0.559 ms, no grouping 0.572 ms, groups of four 0.578 ms (480x832 window).
 #ifndef REGENVC_EXP_GROUP
-#define REGENVC_EXP_GROUP 16
+#define REGENVC_EXP_GROUP 8
 #endif
 constexpr int kExpGroup = REGENVC_EXP_GROUP;
 template <uint32_t kMask>
