@@ -109,3 +109,43 @@ def test_output_projection_argument_checks():
     assert L.regenvc_out_project(None, wd.data_ptr(), None, y.data_ptr(), N, h, D, None) == binding.ERR_NULL_POINTER
     assert L.regenvc_out_project(od.data_ptr(), wd.data_ptr(), None, y.data_ptr(), 0, h, D, None) == binding.ERR_BAD_SHAPE
     assert L.regenvc_out_project(od.data_ptr() + 2, wd.data_ptr(), None, y.data_ptr(), N - 1, h, D, None) == binding.ERR_MISALIGNED
+
+
+def test_a_sustained_loop_of_the_block_chain_stays_bit_exact():
+    """One and a half seconds of the whole chain at the 480x832 window shape (producer -> attention on its operands
+    -> output projection, back to back, long enough to reach the power cap): every repetition must reproduce the
+    first one bit for bit -- Q', K', V't, the attention output and y -- and no bounded wait may expire.  The producer
+    exchanges partial row sums between thread blocks and all three kernels hand buffers over between warps on
+    barriers: a hand-over that only holds on typical timing shows up here as a changed bit."""
+    import time
+
+    w = synth.WORKLOADS["window_480x832"]
+    x, wq, b, gq, gk, eps = (t.to(DEV) if torch.is_tensor(t) else t for t in synth.block_inputs(w))
+    wo, bo = (t.to(DEV) for t in synth.out_proj_inputs(w))
+    N, h = w.n_tokens, w.n_heads
+
+    def chain(q_rot, prepared, out, y):
+        binding.regenvc_qkv_rope_project(x, wq, b, gq, gk, eps, w.T, w.H, w.W, h, w.theta, q_rot=q_rot, prepared=prepared)
+        binding.regenvc_attn_forward_prepared(q_rot, prepared, N, out)
+        binding.regenvc_out_project(out, wo, bo, y)
+
+    def buffers():
+        return (torch.empty((N, h, D), dtype=torch.float16, device=DEV),
+                torch.zeros((binding.regenvc_prepared_bytes(N, h),), dtype=torch.uint8, device=DEV),
+                torch.empty((N, h, D), dtype=torch.bfloat16, device=DEV),
+                torch.empty((N, h * D), dtype=torch.bfloat16, device=DEV))
+
+    first, again = buffers(), buffers()
+    chain(*first)
+    mismatches = torch.zeros((), dtype=torch.int64, device=DEV)
+    t0, reps = time.time(), 0
+    while time.time() - t0 < 1.5:
+        for _ in range(20):
+            chain(*again)
+            for a, f in zip(again, first):
+                mismatches += (a.view(torch.uint8) != f.view(torch.uint8)).sum()
+            reps += 1
+        torch.cuda.synchronize()
+    assert reps >= 40
+    assert int(mismatches.item()) == 0
+    assert binding.regenvc_device_status() == 0
