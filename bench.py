@@ -46,10 +46,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 PAPER_CONTEXT = ("paper: 972 ms per 25-frame window (24 fps) for the WHOLE decoder on 8 consumer-class GPUs; "
                  "it reports no attention-only number")
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the self-attention kernel at the 480x832 window
-# shape, from one ncu capture of that launch (101.3 MB read + 16.8 MB written; the rest of the 33.5 MB output is
+# shape, from one ncu capture of that launch (101.3 MB read + 17.5 MB written; the rest of the 33.5 MB output is
 # still in L2 when the kernel ends).
-ATTN_KERNEL_DRAM_TRAFFIC_BYTES = {"window_480x832": 118.1e6}
+ATTN_KERNEL_DRAM_TRAFFIC_BYTES = {"window_480x832": 118.8e6}
 N_BUFFER_SETS = 4
+KERNEL_BITS = 0  # --kernel: debug bits that force (8) or forbid (16) the attention kernel on pairs of thread blocks
 
 
 def measured_peaks():
@@ -130,6 +131,15 @@ def max_over_ranks(values, dist=None, device="cpu"):
 def whole_job_tflops(world: int, flops_per_step: float, ms_per_step: float) -> float:
     """Weak scaling: every rank processes one window per step; the job's rate is all windows over the slowest rank's time."""
     return world * flops_per_step / (ms_per_step * 1e-3) / 1e12
+
+
+def self_attention_kernel_name(w: synth.Workload, sm_count: int) -> str:
+    """Which kernel the library enqueues for this workload's self-attention call (its rule, restated): long key
+    sequences with at least one full round of work items run on pairs of thread blocks."""
+    n_tiles = -(-w.n_tokens // 128)
+    n_items = -(-w.n_tokens // 256) * w.n_heads
+    pair = KERNEL_BITS == 8 or (KERNEL_BITS == 0 and n_tiles >= 32 and n_items >= sm_count // 2)
+    return ("attn_pair_kernel" if pair else "attn_pipelined_kernel") + " (self-attention)"
 
 
 def step_flops(w: synth.Workload) -> float:
@@ -294,10 +304,14 @@ def time_producer_fusion(binding, w: synth.Workload, dev, stream, n=20):
 
 
 def run_ours(args, w: synth.Workload):
+    global KERNEL_BITS
+    KERNEL_BITS = {"auto": 0, "pair": 8, "single": 16}[args.kernel]
     from paper_2607_28144_b200 import binding, build
 
     build.build()
     rank, world, local, dev, dist, ranks_seen = _setup_ranks(args)
+    if KERNEL_BITS:
+        binding.regenvc_debug_set_phases(3 | KERNEL_BITS)
 
     def barrier():
         if dist is not None:
@@ -340,7 +354,7 @@ def run_ours(args, w: synth.Workload):
         """n launches of the attention kernel of the self-attention call alone (operands already prepared in the
         set's own workspace), rotating over the input sets.  Returns the per-launch times in ms, or the mean
         over the whole loop when per_launch_events is false."""
-        binding.regenvc_debug_set_phases(2)
+        binding.regenvc_debug_set_phases(2 | KERNEL_BITS)
         try:
             if per_launch_events:
                 evs = _events(n)
@@ -363,7 +377,7 @@ def run_ours(args, w: synth.Workload):
             return a.elapsed_time(b) / n
         finally:
             binding.regenvc_set_workspace(None)
-            binding.regenvc_debug_set_phases(3)
+            binding.regenvc_debug_set_phases(3 | KERNEL_BITS)
 
     with torch.cuda.stream(stream):
         for i in range(max(args.warmup, 3)):
@@ -409,13 +423,13 @@ def run_ours(args, w: synth.Workload):
         attn_times = kernel_only_loop(n_k, True)
         burst_sampler.stop()
         attn_ms, attn_ms_best = statistics.mean(attn_times), min(attn_times)
-        binding.regenvc_debug_set_phases(1)
+        binding.regenvc_debug_set_phases(1 | KERNEL_BITS)
         evp = _events(n_k)
         for i, (a, b) in enumerate(evp):
             a.record(stream)
             self_call(sets[i % N_BUFFER_SETS])
             b.record(stream)
-        binding.regenvc_debug_set_phases(3)
+        binding.regenvc_debug_set_phases(3 | KERNEL_BITS)
         torch.cuda.synchronize()
         prep_ms = statistics.mean(a.elapsed_time(b) for a, b in evp)
 
@@ -533,7 +547,7 @@ def run_ours(args, w: synth.Workload):
             "clocks": sampler.summary(),
             # the kernel timed alone (isolated launches after a pause, rotating input sets) against the burst
             # figure of the measured cuBLAS bf16 peak: frac = achieved / peak, achieved = flops / kernel_ms_mean
-            "roofline": {"bound": "tensor", "kernel": "attn_pipelined_kernel (self-attention)",
+            "roofline": {"bound": "tensor", "kernel": self_attention_kernel_name(w, torch.cuda.get_device_properties(dev).multi_processor_count),
                          "achieved": achieved, "peak": burst_peak, "unit": "TFLOP/s", "frac": achieved / burst_peak,
                          "peak_source": f"{peak_kind} cuBLAS bf16 burst (kernel timed alone; fp16 and bf16 operands "
                                         f"run at the same rate)",
@@ -703,6 +717,9 @@ def main():
                     help="spread ONE window over U*R = --gpus ranks as Ulysses x Ring (the paper's decomposition)")
     ap.add_argument("--sustain-seconds", type=float, default=4.0,
                     help="length of the sustained leg (the step loop repeated under the power cap); 0 skips it")
+    ap.add_argument("--kernel", choices=["auto", "pair", "single"], default="auto",
+                    help="auto: the library's own choice of self-attention kernel; pair / single: always the kernel "
+                         "on pairs of thread blocks / always one thread block per work item (for profiles)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-producer", action="store_true", help="skip the producer-fusion leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")

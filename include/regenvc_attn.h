@@ -321,8 +321,13 @@ int regenvc_device_status(void* stream, int* status_out);
  * call), which lets a benchmark time the attention kernel alone.  Bit 2 (value
  * 4, together with bit 0 and/or 1) makes calls with short key sequences use
  * one thread block per work item instead of the persistent form they
- * normally take (same results; for measuring the difference).  Returns
- * REGENVC_ERR_BAD_SHAPE for a mask outside 1..7 or without bit 0 and bit 1.
+ * normally take (same results; for measuring the difference).  Bit 3 (value
+ * 8) sends every call to the attention kernel that runs on pairs of thread
+ * blocks, which the library otherwise picks for long key sequences only, bit
+ * 4 (value 16) keeps every call away from it (same results within rounding
+ * of the split into key-range pieces; for tests and for measuring the
+ * difference).  Returns REGENVC_ERR_BAD_SHAPE for a mask outside 1..31,
+ * without bit 0 and bit 1, or with both bit 3 and bit 4.
  */
 int regenvc_debug_set_phases(int mask);
 

@@ -399,7 +399,8 @@ def regenvc_kernel_launch_count() -> int:
 
 
 def regenvc_debug_set_phases(mask: int):
-    """Profiling aid: 1 = preparation pass only, 2 = attention kernel only, 3 = both (default)."""
+    """Profiling aid: 1 = preparation pass only, 2 = attention kernel only, 3 = both (default); + 4: no persistent
+    form for short key sequences; + 8 / + 16: always / never the kernel on pairs of thread blocks."""
     _check(lib().regenvc_debug_set_phases(mask))
 
 

@@ -123,6 +123,7 @@ int device_state(int* dev_out, DeviceState** st_out) {
                 g_encode = (EncodeTiledFn)fn;
             }
             CUDA_TRY(configure_attn_pipelined());
+            CUDA_TRY(configure_attn_pair());
             CUDA_TRY(configure_qkv_project_pair());
             CUDA_TRY(configure_out_project());
             CUDA_TRY(configure_attn_persistent());
@@ -204,10 +205,10 @@ int rope_table(DeviceState& st, int T, int H, int W, float theta, const float2**
 }
 
 int make_tmap(CUtensorMap* m, void* base, uint64_t inner, uint64_t outer, uint64_t row_bytes,
-              CUtensorMapDataType type = CU_TENSOR_MAP_DATA_TYPE_FLOAT16) {
+              CUtensorMapDataType type = CU_TENSOR_MAP_DATA_TYPE_FLOAT16, int box_rows = 128) {
     const cuuint64_t gdim[2] = {inner, outer};
     const cuuint64_t gstride[1] = {row_bytes};
-    const cuuint32_t box[2] = {64, 128};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode(m, type, 2, base, gdim, gstride, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -279,11 +280,20 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
         if (rc != REGENVC_OK) return rc;
     }
 
+    // Which attention kernel.  Long key sequences with at least one full round of work items go to the kernel on pairs
+    // of CTAs (a pair per item, each CTA one query tile and half of every K' / V't tile: about 3 % faster per key
+    // tile, but its fixed cost per item is paid per 128 rows); short key sequences with query tiles in operand form
+    // to the persistent kernel; everything else to one CTA per item.  Debug bits 8 / 16 force / forbid the first.
+    const int n_tiles = kv_pad / kTile;
+    const int n_items = ((n_q + 2 * kTile - 1) / (2 * kTile)) * n_heads;
+    const bool use_pair = (tl_phases & 8) || (!(tl_phases & 16) && n_tiles >= kPairMinTiles && n_items >= st->sm_count / 2);
+    const int kv_box_rows = use_pair ? 64 : 128;
     CUtensorMap tmap_k, tmap_v;
     rc = make_tmap(&tmap_k, kp, kHeadDim, (uint64_t)n_heads * kv_pad, kHeadDim * sizeof(__half),
-                   qk_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
+                   qk_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, kv_box_rows);
     if (rc != REGENVC_OK) return rc;
-    rc = make_tmap(&tmap_v, vt, (uint64_t)kv_pad, (uint64_t)n_heads * kHeadDim, (uint64_t)kv_pad * sizeof(__half));
+    rc = make_tmap(&tmap_v, vt, (uint64_t)kv_pad, (uint64_t)n_heads * kHeadDim, (uint64_t)kv_pad * sizeof(__half),
+                   CU_TENSOR_MAP_DATA_TYPE_FLOAT16, kv_box_rows);
     if (rc != REGENVC_OK) return rc;
 
     PrepParams pp;
@@ -321,11 +331,10 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)kHeadDim));
     ap.status = st->status;
     ap.sm_count = st->sm_count;
-    // Work decomposition: one CTA per (head, 256 query rows).  The items of the last, incomplete wave are cut
-    // along the key axis into split_k pieces each so that the pieces fill the SMs; a merge kernel combines them.
-    const int n_tiles = kv_pad / kTile;
+    // Work decomposition: one CTA (or pair of CTAs) per (head, 256 query rows).  The items of the last, incomplete
+    // wave are cut along the key axis into split_k pieces each so that the pieces fill the SMs; a merge kernel
+    // combines them.
     ap.pairs_per_head = (n_q + 2 * kTile - 1) / (2 * kTile);
-    const int n_items = ap.pairs_per_head * n_heads;
     ap.n_full_items = n_items;
     ap.split_k = 1;
     ap.tiles_per_piece = n_tiles;
@@ -333,10 +342,11 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     ap.part_ml = reinterpret_cast<float2*>(ap.part_o + (size_t)kMaxPieceCtas * 2 * kTile * kHeadDim);
     // Short key sequences with query tiles in operand form: one persistent CTA per SM walks over the items and
     // overlaps their fixed costs (no key-range pieces in that form).
-    const bool persistent = q_operand && blk.tok_o == nullptr && n_tiles <= kPersistentMaxTiles && !(tl_phases & 4);
-    const int rem = n_items % st->sm_count;
+    const bool persistent = !use_pair && q_operand && blk.tok_o == nullptr && n_tiles <= kPersistentMaxTiles && !(tl_phases & 4);
+    const int slots = use_pair ? st->sm_count / 2 : st->sm_count;   // work items that run at a time
+    const int rem = n_items % slots;
     if (!persistent && rem > 0 && st->sm_count <= kMaxPieceCtas && blk.tok_o == nullptr) {
-        int k = st->sm_count / rem;
+        int k = slots / rem;
         if (k > 8) k = 8;
         if (k > n_tiles / 4) k = n_tiles / 4;
         if (k >= 2) {
@@ -367,7 +377,8 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
         }
         CUDA_TRY(launch_attn_persistent(tmap_k, tmap_v, tmap_out, tmap_q, ap, n_ctas, stream));
     } else {
-        CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, stream));
+        if (use_pair) CUDA_TRY(launch_attn_pair(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, stream));
+        else CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, stream));
     }
     launched();
     if (ap.split_k > 1) {
@@ -881,7 +892,7 @@ int regenvc_device_status(void* stream, int* status_out) {
 }
 
 int regenvc_debug_set_phases(int mask) {
-    if (mask < 1 || mask > 7 || !(mask & 3)) return REGENVC_ERR_BAD_SHAPE;
+    if (mask < 1 || mask > 31 || !(mask & 3) || (mask & 24) == 24) return REGENVC_ERR_BAD_SHAPE;
     tl_phases = mask;
     return REGENVC_OK;
 }

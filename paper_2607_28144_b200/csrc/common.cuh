@@ -154,6 +154,12 @@ constexpr int kPersistentMaxTiles = 8;
 cudaError_t configure_attn_persistent();
 cudaError_t launch_attn_persistent(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
                                    const CUtensorMap& tmap_q, const AttnParams& p, int n_ctas, cudaStream_t stream);
+// Kernel on pairs of CTAs (attn_pair.cu): one cluster of two per work item, tmap_k / tmap_v with boxes of 64 rows.
+// The host uses it for key sequences of at least kPairMinTiles tiles.
+constexpr int kPairMinTiles = 32;
+cudaError_t configure_attn_pair();
+cudaError_t launch_attn_pair(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
+                             const CUtensorMap* tmap_q, const AttnParams& p, cudaStream_t stream);
 cudaError_t configure_attn_pipelined();   // once per device: register hand-over check, large dynamic shared memory
 cudaError_t launch_merge_partials(const MergeParams& p, cudaStream_t stream);
 cudaError_t launch_merge_token_partials(const TokenMergeParams& p, cudaStream_t stream);

@@ -1,0 +1,119 @@
+"""The attention kernel on pairs of thread blocks (the library picks it for long key sequences) against the oracle
+at sizes the oracle finishes quickly: the calling thread's debug switch sends every call there, and the parity cases
+of the other test files are run once more under it -- ragged tails, odd tile counts (a pair whose second query tile
+does not exist), key-range pieces with their merge, the block-wise partial/merge pair, operands written by a producer,
+and the inputs that make the optimistic pass saturate so that the pair runs its careful second pass (in one of its two
+thread blocks only, in one work item only, along the whole sequence).  At the 480x832 window shape, where the library
+picks the kernel by itself, the two kernels' outputs are compared with each other."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import test_gpu_blockwise
+import test_gpu_parity
+import test_gpu_prepared
+from paper_2607_28144_b200 import binding, synth
+from parity_util import assert_parity
+
+pytestmark = pytest.mark.gpu
+FORCE_PAIR, FORBID_PAIR, DEFAULT = 3 | 8, 3 | 16, 3
+
+
+@pytest.fixture
+def pair_kernel():
+    binding.regenvc_debug_set_phases(FORCE_PAIR)
+    yield
+    binding.regenvc_debug_set_phases(DEFAULT)
+
+
+@pytest.mark.parametrize("grid,h", [((1, 1, 1), 1), ((2, 8, 8), 2), ((1, 11, 13), 3), ((3, 9, 10), 2), ((1, 16, 25), 1)])
+def test_small_self_attention_shapes(pair_kernel, grid, h):
+    test_gpu_parity.test_self_attention_small_shapes(grid, h)
+
+
+@pytest.mark.parametrize("grid,h", [((7, 16, 16), 2), ((1, 25, 44), 3), ((2, 37, 29), 1), ((1, 40, 64), 5)])
+def test_key_range_pieces_and_merge(pair_kernel, grid, h):
+    test_gpu_parity.test_self_attention_with_split_key_pieces(grid, h)
+
+
+@pytest.mark.parametrize("n_q,n_kv,h", [(130, 1, 1), (257, 127, 2), (300, 129, 3), (64, 769, 2), (1100, 1300, 2)])
+def test_cross_attention_shapes(pair_kernel, n_q, n_kv, h):
+    test_gpu_parity.test_cross_attention(n_q, n_kv, h)
+
+
+@pytest.mark.parametrize("scale", [0.5, 2.0])
+def test_score_range(pair_kernel, scale):
+    test_gpu_parity.test_self_attention_score_range(scale)
+
+
+def test_closed_forms(pair_kernel):
+    test_gpu_parity.test_zero_queries_give_column_mean_everywhere()
+    test_gpu_parity.test_constant_value_rows_come_back_exactly()
+    test_gpu_parity.test_position_probe_values()
+    test_gpu_parity.test_dominating_key_and_large_scores()
+
+
+@pytest.mark.parametrize("growth", [3.0, 12.0, 40.0])
+def test_second_pass_along_the_whole_sequence(pair_kernel, growth):
+    test_gpu_parity.test_scores_that_grow_along_the_sequence_force_reference_updates(growth)
+
+
+@pytest.mark.parametrize("key,amp", [(128 + 4, 3.5), (128 + 13, 5.0), (256 + 37, 4.0), (256 + 28, 3.5)])
+def test_second_pass_after_one_jump(pair_kernel, key, amp):
+    test_gpu_parity.test_one_key_far_above_the_reference_of_the_earlier_tiles(key, amp)
+
+
+@pytest.mark.parametrize("key", [900, 1290])
+def test_second_pass_in_one_work_item_and_one_block_of_its_pair(pair_kernel, key):
+    # the saturating query rows 300..329 lie in the SECOND query tile of the item 256..511: only that thread block of
+    # the pair sees the saturation, both must run the second pass
+    test_gpu_parity.test_a_saturation_in_one_work_item_only(key)
+
+
+@pytest.mark.parametrize("case", [0, 1, 2, 3])
+def test_blockwise_partials_and_merge(pair_kernel, case):
+    params = [((2, 9, 14), 2, (0, 252), [0, 126, 252]), ((3, 10, 13), 3, (0, 390), [0, 100, 257, 390]),
+              ((2, 16, 20), 2, (160, 480), [0, 320, 640]), ((1, 30, 40), 1, (1000, 1200), [0, 1, 129, 700, 1200])]
+    test_gpu_blockwise.test_merged_blocks_equal_unsharded_attention(*params[case])
+
+
+@pytest.mark.parametrize("grid,h", [((2, 3, 4), 1), ((3, 7, 13), 2), ((2, 16, 20), 4)])
+def test_operands_written_by_a_producer(pair_kernel, grid, h):
+    test_gpu_prepared.test_attention_on_producer_written_operands(grid, h)
+
+
+def test_debug_switch_argument_checks():
+    L = binding.lib()
+    assert L.regenvc_debug_set_phases(8) == binding.ERR_BAD_SHAPE           # neither pass selected
+    assert L.regenvc_debug_set_phases(3 | 8 | 16) == binding.ERR_BAD_SHAPE  # always and never
+    assert L.regenvc_debug_set_phases(32 | 3) == binding.ERR_BAD_SHAPE
+    assert L.regenvc_debug_set_phases(DEFAULT) == 0
+
+
+def test_the_library_picks_the_pair_kernel_at_the_window_shape_and_both_kernels_agree():
+    """480x832 window, 12 heads: 516 work items of 86 key tiles.  By itself the library takes the kernel on pairs
+    (its output is what test_gpu_full_size.py compares with the oracle); forced the other way the output must agree
+    within two bf16 roundings of the split into key-range pieces."""
+    w = synth.WORKLOADS["window_480x832"]
+    q, k, v = synth.self_inputs(w)
+    dev = torch.device("cuda:0")
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    outs = {}
+    try:
+        for name, mask in (("default", DEFAULT), ("pair", FORCE_PAIR), ("single", FORBID_PAIR)):
+            binding.regenvc_debug_set_phases(mask)
+            out = torch.full_like(qd, float("nan"))
+            binding.regenvc_attn_forward(qd, kd, vd, out, w.T, w.H, w.W, w.theta)
+            assert binding.regenvc_device_status() == 0
+            outs[name] = out.float().cpu()
+    finally:
+        binding.regenvc_debug_set_phases(DEFAULT)
+    assert torch.equal(outs["default"], outs["pair"]), "the default call did not take the kernel on pairs"
+    diff = (outs["pair"] - outs["single"]).abs()
+    assert torch.isfinite(diff).all()
+    assert float(diff.max()) <= 2.0 ** -7 * float(v.float().abs().max())
+    assert float(diff.sum() / outs["single"].abs().sum()) <= 1.5e-3
+    rows = np.unique(np.concatenate([np.arange(0, 8), np.arange(w.n_tokens - 8, w.n_tokens)]))
+    ref = oracle.self_attn_head(synth.bits(q), synth.bits(k), synth.bits(v), w.T, w.H, w.W, 5, w.theta, rows=rows)
+    assert_parity(outs["pair"][rows, 5].double().numpy(), ref, float(v.float().abs().max()), "pair kernel, head 5")
