@@ -48,6 +48,7 @@ struct DeviceState {
     bool checked = false, supported = false;
     int* status = nullptr;
     int sm_count = 0;
+    int pair_clusters = 0;   // pairs of CTAs of the attention kernel on pairs that the device holds at a time
     std::vector<RopeEntry> ropes;
     std::map<std::thread::id, Workspace> workspace;
     std::map<std::thread::id, std::vector<Buf>> staging;  // q, k, v, out
@@ -123,7 +124,7 @@ int device_state(int* dev_out, DeviceState** st_out) {
                 g_encode = (EncodeTiledFn)fn;
             }
             CUDA_TRY(configure_attn_pipelined());
-            CUDA_TRY(configure_attn_pair());
+            CUDA_TRY(configure_attn_pair(&st.pair_clusters));
             CUDA_TRY(configure_qkv_project_pair());
             CUDA_TRY(configure_out_project());
             CUDA_TRY(configure_attn_persistent());
@@ -280,13 +281,16 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
         if (rc != REGENVC_OK) return rc;
     }
 
-    // Which attention kernel.  Long key sequences with at least one full round of work items go to the kernel on pairs
-    // of CTAs (a pair per item, each CTA one query tile and half of every K' / V't tile: about 3 % faster per key
-    // tile, but its fixed cost per item is paid per 128 rows); short key sequences with query tiles in operand form
-    // to the persistent kernel; everything else to one CTA per item.  Debug bits 8 / 16 force / forbid the first.
+    // Which attention kernel.  Long key sequences with at least one full round of work items go to the persistent
+    // kernel on pairs of CTAs (a pair per item, each CTA one query tile and half of every K' / V't tile; the pairs walk
+    // over the items, so the fixed cost of an item overlaps the end of the one before it); short key sequences with
+    // query tiles in operand form to the persistent kernel for those; everything else to one CTA per item.  Debug bits
+    // 8 / 16 force / forbid the first.  A launch of the kernel on pairs covers a bounded number of units per pair.
     const int n_tiles = kv_pad / kTile;
     const int n_items = ((n_q + 2 * kTile - 1) / (2 * kTile)) * n_heads;
-    const bool use_pair = (tl_phases & 8) || (!(tl_phases & 16) && n_tiles >= kPairMinTiles && n_items >= st->sm_count / 2);
+    const bool pair_fits = (long long)n_items + 8LL * st->pair_clusters <= (long long)st->pair_clusters * kPairMaxItemsPerPair;
+    const bool use_pair = pair_fits && ((tl_phases & 8) || (!(tl_phases & 16) && n_tiles >= kPairMinTiles &&
+                                                            n_items >= st->pair_clusters));
     const int kv_box_rows = use_pair ? 64 : 128;
     CUtensorMap tmap_k, tmap_v;
     rc = make_tmap(&tmap_k, kp, kHeadDim, (uint64_t)n_heads * kv_pad, kHeadDim * sizeof(__half),
@@ -343,7 +347,7 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     // Short key sequences with query tiles in operand form: one persistent CTA per SM walks over the items and
     // overlaps their fixed costs (no key-range pieces in that form).
     const bool persistent = !use_pair && q_operand && blk.tok_o == nullptr && n_tiles <= kPersistentMaxTiles && !(tl_phases & 4);
-    const int slots = use_pair ? st->sm_count / 2 : st->sm_count;   // work items that run at a time
+    const int slots = use_pair ? st->pair_clusters : st->sm_count;   // work items that run at a time
     const int rem = n_items % slots;
     if (!persistent && rem > 0 && st->sm_count <= kMaxPieceCtas && blk.tok_o == nullptr) {
         int k = slots / rem;
@@ -377,7 +381,7 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
         }
         CUDA_TRY(launch_attn_persistent(tmap_k, tmap_v, tmap_out, tmap_q, ap, n_ctas, stream));
     } else {
-        if (use_pair) CUDA_TRY(launch_attn_pair(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, stream));
+        if (use_pair) CUDA_TRY(launch_attn_pair(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, st->pair_clusters, stream));
         else CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, stream));
     }
     launched();

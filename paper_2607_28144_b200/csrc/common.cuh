@@ -154,12 +154,15 @@ constexpr int kPersistentMaxTiles = 8;
 cudaError_t configure_attn_persistent();
 cudaError_t launch_attn_persistent(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
                                    const CUtensorMap& tmap_q, const AttnParams& p, int n_ctas, cudaStream_t stream);
-// Kernel on pairs of CTAs (attn_pair.cu): one cluster of two per work item, tmap_k / tmap_v with boxes of 64 rows.
-// The host uses it for key sequences of at least kPairMinTiles tiles.
+// Kernel on pairs of CTAs (attn_pair.cu): a persistent grid of clusters of two walks over the work items; tmap_k /
+// tmap_v with boxes of 64 rows.  The host uses it for key sequences of at least kPairMinTiles tiles.
+// configure_attn_pair reports how many pairs the device holds at a time (the grid size); a launch covers at most
+// that many times kPairMaxItemsPerPair units of work.
 constexpr int kPairMinTiles = 32;
-cudaError_t configure_attn_pair();
+constexpr int kPairMaxItemsPerPair = 256;
+cudaError_t configure_attn_pair(int* max_clusters);
 cudaError_t launch_attn_pair(const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, const CUtensorMap& tmap_out,
-                             const CUtensorMap* tmap_q, const AttnParams& p, cudaStream_t stream);
+                             const CUtensorMap* tmap_q, const AttnParams& p, int max_clusters, cudaStream_t stream);
 cudaError_t configure_attn_pipelined();   // once per device: register hand-over check, large dynamic shared memory
 cudaError_t launch_merge_partials(const MergeParams& p, cudaStream_t stream);
 cudaError_t launch_merge_token_partials(const TokenMergeParams& p, cudaStream_t stream);

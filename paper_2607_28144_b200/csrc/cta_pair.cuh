@@ -90,6 +90,12 @@ __device__ __forceinline__ void mbar_arrive_peer(uint32_t bar) {
 __device__ __forceinline__ void st_shared_peer(uint32_t addr, uint32_t v) {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
+// One 32-bit word from the shared memory of either CTA of the pair (shared::cluster address).
+__device__ __forceinline__ uint32_t ld_shared_peer(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
 }  // namespace
 
 }  // namespace regenvc
