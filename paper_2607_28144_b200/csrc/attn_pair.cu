@@ -70,6 +70,10 @@ static_assert(kPairAttnSmem <= 232448, "shared memory of one SM");
 constexpr uint32_t kPColS = 0, kPColO = 384;   // tensor-memory columns: three score buffers, then the accumulator
 constexpr int kQueryWarp0 = kTmaWarp + 1;      // first of the two query warps
 constexpr int kQueryThreads = 64;
+#ifndef REGENVC_PAIR_ROUNDS
+#define REGENVC_PAIR_ROUNDS 12
+#endif
+constexpr int kPairMaxPersistentRounds = REGENVC_PAIR_ROUNDS;   // units per pair up to which the grid is persistent
 
 struct PairBarriers {
     uint64_t kv_full[kPairStages];
@@ -447,7 +451,10 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
           int k = 0;
           for (int i = walk.from(pass, 0); ok && i >= 0; i = walk.from(pass, i + 1), ++k) {
               const int n = n_before + k;
-              ok = mbar_wait(smem_u32(&bar->stage_full[n & 1]), (n >> 1) & 1, ctl);
+              // one lane polls, with pauses: an item takes a hundred thousand cycles, and a polling warp takes issue
+              // slots from the softmax warps of its scheduler; the other warp sleeps at the named barrier
+              if (qtid == 0) ok = mbar_wait_paused(smem_u32(&bar->stage_full[n & 1]), (n >> 1) & 1, ctl, 200);
+              __syncwarp();
               if (query_warps_any(!ok)) {   // the two warps stay together: they share named barriers below
                   ok = false;
                   break;
@@ -465,14 +472,15 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
               query_warps_barrier();
               if (i_next >= 0) prepare_next();
           }
-          // a second pass stores some tiles again: this pass's stores are complete before it starts (and before exit)
-          if (qtid == 0) tma_store_wait_all();
         }
         __syncwarp();
         if (pass == 0) {
             cluster_sync_all();   // both CTAs' masks are final
             if (!walk.any_marked()) break;
             n_before = walk.n_local;
+            // the second pass stores some tiles again: the first pass's stores of this thread are complete (not just
+            // done reading shared memory) before it issues another one
+            if (tid == kQueryWarp0 * 32) tma_store_wait_all();
         }
       }
     } else {
@@ -786,7 +794,11 @@ cudaError_t launch_attn_pair(const CUtensorMap& tmap_k, const CUtensorMap& tmap_
                              const CUtensorMap* tmap_q, const AttnParams& p, int max_clusters, cudaStream_t stream) {
     const int n_items = p.pairs_per_head * p.h;
     const int n_units = p.n_full_items + (n_items - p.n_full_items) * p.split_k;
-    const int n_clusters = n_units < max_clusters ? n_units : max_clusters;
+    // A persistent grid hands the units out statically (pair c: c, c + G, ...), which saves the fixed cost per unit but
+    // cannot even out pairs that run at different speeds; with many units per pair the hardware's own scheduling of one
+    // cluster per unit balances better than the overlap saves (measured at 27 and 66 units per pair).
+    const bool persistent = n_units <= kPairMaxPersistentRounds * max_clusters;
+    const int n_clusters = (!persistent || n_units < max_clusters) ? n_units : max_clusters;
     if (n_clusters < 1 || (long long)n_clusters * kPairMaxItemsPerPair < n_units) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * (unsigned)n_clusters);

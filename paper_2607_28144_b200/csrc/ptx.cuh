@@ -87,6 +87,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
     }
 }
 
+// The same for one thread that expects to wait long (tens of microseconds): it pauses `pause_ns` between the polls,
+// so that its warp leaves the issue slots to the others.  Same limit, same error behaviour.
+__device__ __forceinline__ bool mbar_wait_paused(uint32_t bar, uint32_t parity, const WaitCtl& ctl, uint32_t pause_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    while (true) {
+        __nanosleep(pause_ns);
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*ctl.abort_flag) return false;
+        if (global_timer_ns() - t0 > ctl.limit_ns) {
+            *ctl.abort_flag = 1;
+            atomicCAS(ctl.status, 0, ctl.code);
+            return false;
+        }
+    }
+}
+
 // ------------------------------------------------------------------ shared-memory scalars by 32-bit address
 __device__ __forceinline__ void sts_f32(uint32_t addr, float v) {
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
