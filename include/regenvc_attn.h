@@ -326,8 +326,11 @@ int regenvc_device_status(void* stream, int* status_out);
  * blocks, which the library otherwise picks for long key sequences only, bit
  * 4 (value 16) keeps every call away from it (same results within rounding
  * of the split into key-range pieces; for tests and for measuring the
- * difference).  Returns REGENVC_ERR_BAD_SHAPE for a mask outside 1..31,
- * without bit 0 and bit 1, or with both bit 3 and bit 4.
+ * difference).  Bit 5 (value 32) sends every call to that kernel too, with a
+ * grid of two pairs of thread blocks only, so that even a small call makes
+ * each pair walk over many work items (for tests of that walk).  Returns
+ * REGENVC_ERR_BAD_SHAPE for a mask outside 1..63, without bit 0 and bit 1, or
+ * with bit 4 together with bit 3 or bit 5.
  */
 int regenvc_debug_set_phases(int mask);
 

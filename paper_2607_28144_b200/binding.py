@@ -400,7 +400,8 @@ def regenvc_kernel_launch_count() -> int:
 
 def regenvc_debug_set_phases(mask: int):
     """Profiling aid: 1 = preparation pass only, 2 = attention kernel only, 3 = both (default); + 4: no persistent
-    form for short key sequences; + 8 / + 16: always / never the kernel on pairs of thread blocks."""
+    form for short key sequences; + 8 / + 16: always / never the kernel on pairs of thread blocks; + 32: always that
+    kernel, on a grid of two pairs that walk over all work items."""
     _check(lib().regenvc_debug_set_phases(mask))
 
 

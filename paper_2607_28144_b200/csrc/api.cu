@@ -285,11 +285,12 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     // kernel on pairs of CTAs (a pair per item, each CTA one query tile and half of every K' / V't tile; the pairs walk
     // over the items, so the fixed cost of an item overlaps the end of the one before it); short key sequences with
     // query tiles in operand form to the persistent kernel for those; everything else to one CTA per item.  Debug bits
-    // 8 / 16 force / forbid the first.  A launch of the kernel on pairs covers a bounded number of units per pair.
+    // 8 / 16 force / forbid the first (32: force it with a grid of two pairs only, so that small shapes take many
+    // items per pair).  A launch of the kernel on pairs covers a bounded number of units per pair.
     const int n_tiles = kv_pad / kTile;
     const int n_items = ((n_q + 2 * kTile - 1) / (2 * kTile)) * n_heads;
     const bool pair_fits = (long long)n_items + 8LL * st->pair_clusters <= (long long)st->pair_clusters * kPairMaxItemsPerPair;
-    const bool use_pair = pair_fits && ((tl_phases & 8) || (!(tl_phases & 16) && n_tiles >= kPairMinTiles &&
+    const bool use_pair = pair_fits && ((tl_phases & 40) || (!(tl_phases & 16) && n_tiles >= kPairMinTiles &&
                                                             n_items >= st->pair_clusters));
     const int kv_box_rows = use_pair ? 64 : 128;
     CUtensorMap tmap_k, tmap_v;
@@ -381,7 +382,8 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
         }
         CUDA_TRY(launch_attn_persistent(tmap_k, tmap_v, tmap_out, tmap_q, ap, n_ctas, stream));
     } else {
-        if (use_pair) CUDA_TRY(launch_attn_pair(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, st->pair_clusters, stream));
+        if (use_pair) CUDA_TRY(launch_attn_pair(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap,
+                                                    (tl_phases & 32) ? -2 : st->pair_clusters, stream));
         else CUDA_TRY(launch_attn_pipelined(tmap_k, tmap_v, tmap_out, q_operand ? &tmap_q : nullptr, ap, stream));
     }
     launched();
@@ -896,7 +898,7 @@ int regenvc_device_status(void* stream, int* status_out) {
 }
 
 int regenvc_debug_set_phases(int mask) {
-    if (mask < 1 || mask > 31 || !(mask & 3) || (mask & 24) == 24) return REGENVC_ERR_BAD_SHAPE;
+    if (mask < 1 || mask > 63 || !(mask & 3) || (mask & 24) == 24 || (mask & 48) == 48) return REGENVC_ERR_BAD_SHAPE;
     tl_phases = mask;
     return REGENVC_OK;
 }

@@ -797,7 +797,10 @@ cudaError_t launch_attn_pair(const CUtensorMap& tmap_k, const CUtensorMap& tmap_
     // A persistent grid hands the units out statically (pair c: c, c + G, ...), which saves the fixed cost per unit but
     // cannot even out pairs that run at different speeds; with many units per pair the hardware's own scheduling of one
     // cluster per unit balances better than the overlap saves (measured at 27 and 66 units per pair).
-    const bool persistent = n_units <= kPairMaxPersistentRounds * max_clusters;
+    // (max_clusters < 0, a test aid: a grid of at most -max_clusters pairs that always walks)
+    const bool walk_always = max_clusters < 0;
+    if (walk_always) max_clusters = -max_clusters;
+    const bool persistent = walk_always || n_units <= kPairMaxPersistentRounds * max_clusters;
     const int n_clusters = (!persistent || n_units < max_clusters) ? n_units : max_clusters;
     if (n_clusters < 1 || (long long)n_clusters * kPairMaxItemsPerPair < n_units) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};

@@ -2,9 +2,12 @@
 at sizes the oracle finishes quickly: the calling thread's debug switch sends every call there, and the parity cases
 of the other test files are run once more under it -- ragged tails, odd tile counts (a pair whose second query tile
 does not exist), key-range pieces with their merge, the block-wise partial/merge pair, operands written by a producer,
-and the inputs that make the optimistic pass saturate so that the pair runs its careful second pass (in one of its two
-thread blocks only, in one work item only, along the whole sequence).  At the 480x832 window shape, where the library
-picks the kernel by itself, the two kernels' outputs are compared with each other."""
+and the inputs that make the optimistic run saturate so that the pair runs the item again carefully (a saturation in
+one of its two thread blocks only, in one work item only, along the whole sequence).  Every case runs twice: with one
+pair per work item, and on a grid of two pairs that walk over all work items (the form large calls take: the next
+item's query tile prepared and its first score tiles issued while the current item finishes, finished tiles written out
+by the query warps, marked items run again after the last one).  At the 480x832 window shape, where the library picks
+the kernel by itself, the two kernels' outputs are compared with each other."""
 import numpy as np
 import pytest
 import torch
@@ -17,12 +20,12 @@ from paper_2607_28144_b200 import binding, synth
 from parity_util import assert_parity
 
 pytestmark = pytest.mark.gpu
-FORCE_PAIR, FORBID_PAIR, DEFAULT = 3 | 8, 3 | 16, 3
+FORCE_PAIR, FORBID_PAIR, TWO_PAIRS_WALK, DEFAULT = 3 | 8, 3 | 16, 3 | 32, 3
 
 
-@pytest.fixture
-def pair_kernel():
-    binding.regenvc_debug_set_phases(FORCE_PAIR)
+@pytest.fixture(params=[FORCE_PAIR, TWO_PAIRS_WALK], ids=["pair_per_item", "two_pairs_walk"])
+def pair_kernel(request):
+    binding.regenvc_debug_set_phases(request.param)
     yield
     binding.regenvc_debug_set_phases(DEFAULT)
 
@@ -71,6 +74,37 @@ def test_second_pass_in_one_work_item_and_one_block_of_its_pair(pair_kernel, key
     test_gpu_parity.test_a_saturation_in_one_work_item_only(key)
 
 
+def test_saturations_in_several_work_items_far_apart(pair_kernel):
+    """Nine work items per head and two heads, eleven key tiles.  Query rows of items 1, 4 and 8 of head 0 and of
+    item 6 of head 1 each point at a late key of their own with a score about 200 log2 units above everything else:
+    those four items saturate in their optimistic run and are run again carefully -- by the walking grid after its
+    last item, in list order, with clean items in between that must keep their first result."""
+    n_q, n_kv, h = 2200, 1300, 2
+    rng = np.random.default_rng(47)
+    q = rng.standard_normal((n_q, h, test_gpu_parity.D)).astype(np.float32)
+    k = rng.standard_normal((n_kv, h, test_gpu_parity.D)).astype(np.float32)
+    cases = [(0, 300, 700), (0, 1100, 1290), (0, 2100, 450), (1, 1600, 1000)]   # head, first query row, key
+    for hd, r0, key in cases:
+        sign = rng.choice([-1.0, 1.0], size=test_gpu_parity.D).astype(np.float32)
+        q[r0:r0 + 20, hd] = 3.5 * sign
+        k[key, hd] = 3.5 * sign
+    q, k, v = synth.from_f32(q), synth.from_f32(k), test_gpu_parity._rand(rng, n_kv, h)
+    gpu = test_gpu_parity.f64(test_gpu_parity.run_gpu_cross(q, k, v))
+    ref = oracle.cross_attention(synth.bits(q), synth.bits(k), synth.bits(v))
+    vmax = float(v.float().abs().max())
+    for hd, r0, key in cases:
+        np.testing.assert_allclose(ref[r0:r0 + 20, hd], np.broadcast_to(test_gpu_parity.f64(v)[key, hd], (20, test_gpu_parity.D)),
+                                   atol=1e-9)
+        assert_parity(gpu[r0:r0 + 20, hd:hd + 1], ref[r0:r0 + 20, hd:hd + 1], vmax, f"saturated rows {r0}.. of head {hd}")
+    assert_parity(gpu, ref, vmax, "four saturating work items of eighteen")
+
+
+@pytest.mark.parametrize("n_q,n_kv,h", [(2300, 100, 3), (3000, 128, 2), (1500, 250, 4)])
+def test_many_work_items_of_one_or_two_key_tiles(pair_kernel, n_q, n_kv, h):
+    # items of a single key tile (and of two): the score stream runs across two item boundaries at a time
+    test_gpu_parity.test_cross_attention(n_q, n_kv, h)
+
+
 @pytest.mark.parametrize("case", [0, 1, 2, 3])
 def test_blockwise_partials_and_merge(pair_kernel, case):
     params = [((2, 9, 14), 2, (0, 252), [0, 126, 252]), ((3, 10, 13), 3, (0, 390), [0, 100, 257, 390]),
@@ -87,7 +121,8 @@ def test_debug_switch_argument_checks():
     L = binding.lib()
     assert L.regenvc_debug_set_phases(8) == binding.ERR_BAD_SHAPE           # neither pass selected
     assert L.regenvc_debug_set_phases(3 | 8 | 16) == binding.ERR_BAD_SHAPE  # always and never
-    assert L.regenvc_debug_set_phases(32 | 3) == binding.ERR_BAD_SHAPE
+    assert L.regenvc_debug_set_phases(3 | 32 | 16) == binding.ERR_BAD_SHAPE  # the walking form of it, and never
+    assert L.regenvc_debug_set_phases(64 | 3) == binding.ERR_BAD_SHAPE
     assert L.regenvc_debug_set_phases(DEFAULT) == 0
 
 
