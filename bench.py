@@ -46,9 +46,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 PAPER_CONTEXT = ("paper: 972 ms per 25-frame window (24 fps) for the WHOLE decoder on 8 consumer-class GPUs; "
                  "it reports no attention-only number")
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the self-attention kernel at the 480x832 window
-# shape, from one ncu capture of that launch (101.3 MB read + 17.5 MB written; the rest of the 33.5 MB output is
+# shape, from one ncu capture of that launch (101.6 MB read + 19.7 MB written; the rest of the 33.5 MB output is
 # still in L2 when the kernel ends).
-ATTN_KERNEL_DRAM_TRAFFIC_BYTES = {"window_480x832": 118.8e6}
+ATTN_KERNEL_DRAM_TRAFFIC_BYTES = {"window_480x832": 121.3e6}
 N_BUFFER_SETS = 4
 KERNEL_BITS = 0  # --kernel: debug bits that force (8) or forbid (16) the attention kernel on pairs of thread blocks
 
