@@ -1,5 +1,6 @@
 // Streaming, warp-specialised tcgen05 attention kernel for sm_100a on PAIRS of CTAs (clusters of two, cta_group::2),
 // persistent: as many pairs as fit on the GPU walk over the work items, pair c taking items c, c + G, c + 2G, ...
+// (calls with many items per pair are launched with one pair per item instead: the host's choice, same kernel).
 //
 // A work item is one head, 256 query rows and a range of key tiles; CTA r of the pair owns the query rows 128 r ..
 // 128 r + 127 (its Q tile, its score / probability / output columns in ITS tensor memory, its softmax warps) and
@@ -70,10 +71,7 @@ static_assert(kPairAttnSmem <= 232448, "shared memory of one SM");
 constexpr uint32_t kPColS = 0, kPColO = 384;   // tensor-memory columns: three score buffers, then the accumulator
 constexpr int kQueryWarp0 = kTmaWarp + 1;      // first of the two query warps
 constexpr int kQueryThreads = 64;
-#ifndef REGENVC_PAIR_ROUNDS
-#define REGENVC_PAIR_ROUNDS 12
-#endif
-constexpr int kPairMaxPersistentRounds = REGENVC_PAIR_ROUNDS;   // units per pair up to which the grid is persistent
+constexpr int kPairMaxPersistentRounds = 12;   // units per pair up to which the grid is persistent
 
 struct PairBarriers {
     uint64_t kv_full[kPairStages];

@@ -12,8 +12,7 @@ namespace {
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// The two halves of that barrier, for warps that have nothing to publish and can do other work in between.
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+// The two halves of that barrier, for warps that can do other work in between.
 // Arrival of warps that have written nothing the other CTA will read (no release: that fence costs several hundred cycles).
 __device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
@@ -86,10 +85,6 @@ __device__ __forceinline__ void mbar_arrive_peer(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-// One 32-bit word into the shared memory of either CTA of the pair (shared::cluster address).
-__device__ __forceinline__ void st_shared_peer(uint32_t addr, uint32_t v) {
-    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
 // One 32-bit word from the shared memory of either CTA of the pair (shared::cluster address).
 __device__ __forceinline__ uint32_t ld_shared_peer(uint32_t addr) {
     uint32_t v;
