@@ -99,6 +99,30 @@ def test_saturations_in_several_work_items_far_apart(pair_kernel):
     assert_parity(gpu, ref, vmax, "four saturating work items of eighteen")
 
 
+def test_saturations_late_in_a_long_list_of_work_items(pair_kernel):
+    """140 work items of three key tiles: on the grid of two pairs each pair walks over 70 of them, so the items that
+    saturate (numbers 77 and 130 of head-major order: the 39th and the 66th of their pairs) are recorded in the second
+    and third word of the pair's mask and found again from there."""
+    n_q, n_kv, h = 256 * 70, 300, 2
+    rng = np.random.default_rng(53)
+    q = rng.standard_normal((n_q, h, test_gpu_parity.D)).astype(np.float32)
+    k = rng.standard_normal((n_kv, h, test_gpu_parity.D)).astype(np.float32)
+    cases = [(1, 256 * 7 + 40, 290), (1, 256 * 60 + 200, 140)]   # head, first query row, key: items 70 + 7, 70 + 60
+    for hd, r0, key in cases:
+        sign = rng.choice([-1.0, 1.0], size=test_gpu_parity.D).astype(np.float32)   # (each case its own direction)
+        q[r0:r0 + 10, hd] = 3.5 * sign
+        k[key, hd] = 3.5 * sign
+    q, k, v = synth.from_f32(q), synth.from_f32(k), test_gpu_parity._rand(rng, n_kv, h)
+    gpu = test_gpu_parity.f64(test_gpu_parity.run_gpu_cross(q, k, v))
+    ref = oracle.cross_attention(synth.bits(q), synth.bits(k), synth.bits(v))
+    vmax = float(v.float().abs().max())
+    for hd, r0, key in cases:
+        np.testing.assert_allclose(ref[r0:r0 + 10, hd], np.broadcast_to(test_gpu_parity.f64(v)[key, hd], (10, test_gpu_parity.D)),
+                                   atol=1e-9)
+        assert_parity(gpu[r0:r0 + 10, hd:hd + 1], ref[r0:r0 + 10, hd:hd + 1], vmax, f"saturated rows {r0}.. of head {hd}")
+    assert_parity(gpu, ref, vmax, "two saturating work items of 140")
+
+
 @pytest.mark.parametrize("n_q,n_kv,h", [(2300, 100, 3), (3000, 128, 2), (1500, 250, 4)])
 def test_many_work_items_of_one_or_two_key_tiles(pair_kernel, n_q, n_kv, h):
     # items of a single key tile (and of two): the score stream runs across two item boundaries at a time
