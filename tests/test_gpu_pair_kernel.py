@@ -141,6 +141,29 @@ def test_operands_written_by_a_producer(pair_kernel, grid, h):
     test_gpu_prepared.test_attention_on_producer_written_operands(grid, h)
 
 
+def test_a_call_that_starts_with_the_error_status_set_ends_by_itself_and_the_next_one_is_normal(pair_kernel):
+    """Seven work items per head, fourteen key tiles.  After a wait has expired (a warp of its own that waits on a
+    barrier nothing completes) the sticky status is set: a call that starts then must give up every wait of its own
+    at once, in every role of both thread blocks of every pair and at every item of the walk, end without help and
+    leave the status for the caller; the call after the status has been read is bit for bit what it was before."""
+    import time
+
+    T, H, W, h = 7, 16, 16, 2
+    rng = np.random.default_rng(61)
+    q, k, v = (test_gpu_parity._rand(rng, T * H * W, h) for _ in range(3))
+    good = test_gpu_parity.run_gpu_self(q, k, v, T, H, W)
+    dev = torch.device("cuda:0")
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    out = torch.zeros_like(qd)
+    binding.regenvc_debug_expire_wait(200)
+    t0 = time.time()
+    binding.regenvc_attn_forward(qd, kd, vd, out, T, H, W)
+    assert binding.regenvc_device_status() == binding.ERR_TIMEOUT
+    assert time.time() - t0 < 5.0
+    assert binding.regenvc_device_status() == 0
+    assert torch.equal(test_gpu_parity.run_gpu_self(q, k, v, T, H, W), good)
+
+
 def test_debug_switch_argument_checks():
     L = binding.lib()
     assert L.regenvc_debug_set_phases(8) == binding.ERR_BAD_SHAPE           # neither pass selected
