@@ -125,6 +125,7 @@ int device_state(int* dev_out, DeviceState** st_out) {
             }
             CUDA_TRY(configure_attn_pipelined());
             CUDA_TRY(configure_attn_pair(&st.pair_clusters));
+            if (st.pair_clusters < 1) st.pair_clusters = st.sm_count / 2 > 0 ? st.sm_count / 2 : 1;
             CUDA_TRY(configure_qkv_project_pair());
             CUDA_TRY(configure_out_project());
             CUDA_TRY(configure_attn_persistent());

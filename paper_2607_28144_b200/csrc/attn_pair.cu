@@ -775,9 +775,13 @@ cudaError_t configure_pair_one(int* max_clusters) {
     cfg.numAttrs = 1;
     int n = 0;
     e = cudaOccupancyMaxActiveClusters(&n, attn_pair_kernel<kQTma>, &cfg);
-    if (e != cudaSuccess) return e;
-    if (n < 1) return cudaErrorInvalidConfiguration;
-    if (*max_clusters == 0 || n < *max_clusters) *max_clusters = n;
+    if (e != cudaSuccess || n < 1) {
+        // no answer: the caller falls back to one pair per two SMs (the grid size only sets how the units are handed
+        // out; any number of pairs computes the same result)
+        (void)cudaGetLastError();
+        n = 0;
+    }
+    if (n > 0 && (*max_clusters == 0 || n < *max_clusters)) *max_clusters = n;
     return cudaSuccess;
 }
 }  // namespace
