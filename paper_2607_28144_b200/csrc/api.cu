@@ -287,12 +287,10 @@ int enqueue(const void* q, const void* k, const void* v, void* out, int n_q, int
     // over the items, so the fixed cost of an item overlaps the end of the one before it); short key sequences with
     // query tiles in operand form to the persistent kernel for those; everything else to one CTA per item.  Debug bits
     // 8 / 16 force / forbid the first (32: force it with a grid of two pairs only, so that small shapes take many
-    // items per pair).  A launch of the kernel on pairs covers a bounded number of units per pair.
+    // items per pair).
     const int n_tiles = kv_pad / kTile;
     const int n_items = ((n_q + 2 * kTile - 1) / (2 * kTile)) * n_heads;
-    const bool pair_fits = (long long)n_items + 8LL * st->pair_clusters <= (long long)st->pair_clusters * kPairMaxItemsPerPair;
-    const bool use_pair = pair_fits && ((tl_phases & 40) || (!(tl_phases & 16) && n_tiles >= kPairMinTiles &&
-                                                            n_items >= st->pair_clusters));
+    const bool use_pair = (tl_phases & 40) || (!(tl_phases & 16) && n_tiles >= kPairMinTiles && n_items >= st->pair_clusters);
     const int kv_box_rows = use_pair ? 64 : 128;
     CUtensorMap tmap_k, tmap_v;
     rc = make_tmap(&tmap_k, kp, kHeadDim, (uint64_t)n_heads * kv_pad, kHeadDim * sizeof(__half),

@@ -38,6 +38,14 @@ constexpr uint32_t kPolyMask = REGENVC_POLY_MASK;
 constexpr uint32_t kIdesc = umma_idesc_f16_f32acc(128, 128);           // fp16 x fp16 -> fp32
 constexpr uint32_t kIdescBf16 = umma_idesc_bf16_f32acc(128, 128);      // bf16 x bf16 -> fp32
 constexpr uint64_t kWaitLimitNs = 500000000ull;   // 0.5 s per wait
+// Headroom of the softmax reference (log2 units): whenever the reference of a row is set from a tile's row maximum it
+// is set this far above it, so the largest probability is 2^-4 and a later score may exceed that maximum by 20 log2
+// units (13.9 nats) instead of 16 before a probability leaves the fp16 range and the item has to be run again.  The
+// cost is at the other end: probabilities more than 10 (instead of 14) log2 units below the largest are subnormal
+// in fp16 and those more than 20 (instead of 24) below it vanish from P.V (never from the fp32 row sum), at most
+// 2^-20 of the largest term each.  With scores of standard deviation 4 nats (the 40-head workload's heads with twice
+// the unit scale) a third of the work items of such a head saturated without the headroom, practically none with it.
+constexpr float kRefMargin = 4.0f;
 
 
 // Values the threads of a row hand each other through shared memory (redo path and epilogue only).

@@ -1,6 +1,6 @@
 // Streaming, warp-specialised tcgen05 attention kernel for sm_100a on PAIRS of CTAs (clusters of two, cta_group::2),
 // persistent: as many pairs as fit on the GPU walk over the work items, pair c taking items c, c + G, c + 2G, ...
-// (calls with many items per pair are launched with one pair per item instead: the host's choice, same kernel).
+// (a call with more items than the pairs' lists can hold is launched with one pair per item instead: same kernel).
 //
 // A work item is one head, 256 query rows and a range of key tiles; CTA r of the pair owns the query rows 128 r ..
 // 128 r + 127 (its Q tile, its score / probability / output columns in ITS tensor memory, its softmax warps) and
@@ -71,7 +71,6 @@ static_assert(kPairAttnSmem <= 232448, "shared memory of one SM");
 constexpr uint32_t kPColS = 0, kPColO = 384;   // tensor-memory columns: three score buffers, then the accumulator
 constexpr int kQueryWarp0 = kTmaWarp + 1;      // first of the two query warps
 constexpr int kQueryThreads = 64;
-constexpr int kPairMaxPersistentRounds = 12;   // units per pair up to which the grid is persistent
 
 struct PairBarriers {
     uint64_t kv_full[kPairStages];
@@ -607,7 +606,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
 #pragma unroll
                   for (int o = 1; o < kSplit; ++o) mx_row = fmaxf(mx_row, xch[row][(part + o) % kSplit]);
                   row_group_barrier(warp & 3);  // everyone has read xch before a later exchange overwrites it
-                  const float m_tile = mx_row * scale;
+                  const float m_tile = mx_row * scale + kRefMargin;
                   const bool raise = m_tile > m_ref;  // always on the first tile (reference starts at -inf)
                   if (j > 0) {
                       // P.V(g - 1) is issued when every warp has handed the previous visit's probabilities over.  Its
@@ -796,13 +795,11 @@ cudaError_t launch_attn_pair(const CUtensorMap& tmap_k, const CUtensorMap& tmap_
                              const CUtensorMap* tmap_q, const AttnParams& p, int max_clusters, cudaStream_t stream) {
     const int n_items = p.pairs_per_head * p.h;
     const int n_units = p.n_full_items + (n_items - p.n_full_items) * p.split_k;
-    // A persistent grid hands the units out statically (pair c: c, c + G, ...), which saves the fixed cost per unit but
-    // cannot even out pairs that run at different speeds; with many units per pair the hardware's own scheduling of one
-    // cluster per unit balances better than the overlap saves (measured at 27 and 66 units per pair).
-    // (max_clusters < 0, a test aid: a grid of at most -max_clusters pairs that always walks)
-    const bool walk_always = max_clusters < 0;
-    if (walk_always) max_clusters = -max_clusters;
-    const bool persistent = walk_always || n_units <= kPairMaxPersistentRounds * max_clusters;
+    // A persistent grid: the pairs the GPU holds at a time, the units handed out statically (pair c: c, c + G, ...).  Only
+    // a call with more units than the pairs' lists can hold gets one cluster per unit instead.
+    // (max_clusters < 0, a test aid: a grid of at most -max_clusters pairs)
+    if (max_clusters < 0) max_clusters = -max_clusters;
+    const bool persistent = (long long)n_units <= (long long)kPairMaxItemsPerPair * max_clusters;
     const int n_clusters = (!persistent || n_units < max_clusters) ? n_units : max_clusters;
     if (n_clusters < 1 || (long long)n_clusters * kPairMaxItemsPerPair < n_units) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};

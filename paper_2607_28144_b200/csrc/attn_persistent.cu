@@ -343,7 +343,7 @@ attn_persistent_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_
 #pragma unroll
                         for (int o = 1; o < kSplit; ++o) mx_row = fmaxf(mx_row, xch[row][(part + o) % kSplit]);
                         row_group_barrier(warp & 3);
-                        const float m_tile = mx_row * scale;
+                        const float m_tile = mx_row * scale + kRefMargin;
                         const bool raise = m_tile > m_ref[t];
                         if (j > 0) {
                             if (ok) ok = mbar_wait_lean(bars, kOffOFull + 8 * t, (visit - 1) & 1, p.status);

@@ -324,7 +324,7 @@ attn_pipelined_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_c
 #pragma unroll
                     for (int o = 1; o < kSplit; ++o) mx_row = fmaxf(mx_row, xch->m[t][row][(part + o) % kSplit]);
                     row_group_barrier(warp & 3);  // everyone has read xch->m before a later redo overwrites it
-                    const float m_tile = mx_row * scale;
+                    const float m_tile = mx_row * scale + kRefMargin;
                     const bool raise = m_tile > m_ref[t];  // always on the first tile (reference starts at -inf)
                     if (j > 0) {
                         if (ok) ok = mbar_wait(smem_u32(&bar->o_full[t]), (v0 + j - 1) & 1, ctl);

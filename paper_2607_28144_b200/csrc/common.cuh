@@ -157,8 +157,8 @@ cudaError_t launch_attn_persistent(const CUtensorMap& tmap_k, const CUtensorMap&
 // Kernel on pairs of CTAs (attn_pair.cu): a persistent grid of clusters of two walks over the work items; tmap_k /
 // tmap_v with boxes of 64 rows.  The host uses it for key sequences of at least kPairMinTiles tiles.
 // configure_attn_pair reports how many pairs the device holds at a time (the grid size); a launch covers at most
-// that many times kPairMaxItemsPerPair units of work.  (max_clusters < 0 in launch_attn_pair, a test aid: a grid of at
-// most -max_clusters pairs that walks whatever the number of units per pair.)
+// that many times kPairMaxItemsPerPair units of work as a persistent grid (more: one cluster per unit).  (max_clusters
+// < 0 in launch_attn_pair, a test aid: a grid of at most -max_clusters pairs.)
 constexpr int kPairMinTiles = 32;
 constexpr int kPairMaxItemsPerPair = 256;
 cudaError_t configure_attn_pair(int* max_clusters);
