@@ -187,7 +187,8 @@ int regenvc_out_project(const void* attn_out, const void* w_o, const void* b_o, 
  *                  (c = log2(e) / sqrt(head_dim), s_m the rotated score)
  *   ml           : device, float pairs [n_q, n_heads]     = (m_row in log2 units, l_row = sum_m 2^(s_m c - m_row))
  * Rotary positions are those of the tokens in the whole grid, so blocks computed on different devices merge
- * exactly.  m_row is a reference at or below the block's row maximum plus 16 (not necessarily the maximum).
+ * exactly.  m_row is a reference between 16 log2 units below and 4 above the block's row maximum (not
+ * necessarily the maximum itself).
  *
  * regenvc_attn_merge(): out[n, a, :] = sum_i w_i o_i / sum_i w_i l_i with w_i = 2^(m_i - max_i m_i), rounded to
  * bf16, for n_parts (1..8) partial results of the same query range.  o_parts / mls are HOST arrays of device
