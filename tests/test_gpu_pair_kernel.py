@@ -164,6 +164,38 @@ def test_a_call_that_starts_with_the_error_status_set_ends_by_itself_and_the_nex
     assert torch.equal(test_gpu_parity.run_gpu_self(q, k, v, T, H, W), good)
 
 
+@pytest.mark.parametrize("h", [296, 297])
+def test_as_many_work_items_as_the_pairs_lists_hold_and_one_head_more(h):
+    """16384 query rows x 296 heads are 18944 work items: on 74 pairs exactly the 256 items a pair's list holds (every
+    word of the mask of items to run again in use); one head more and the call is launched with one pair per item.
+    Short key sequence (200 keys), so the call stays small; the kernel on pairs is forced.  Its output must equal the
+    default kernel's bit for bit (same arithmetic in the same order) and the oracle's on sampled rows of two heads."""
+    n_q, n_kv = 16384, 200
+    dev = torch.device("cuda:0")
+    g = torch.Generator(device=dev).manual_seed(h)
+    q = torch.randn((n_q, h, 128), device=dev, generator=g).to(torch.bfloat16)
+    k = torch.randn((n_kv, h, 128), device=dev, generator=g).to(torch.bfloat16)
+    v = torch.randn((n_kv, h, 128), device=dev, generator=g).to(torch.bfloat16)
+    outs = {}
+    try:
+        for name, mask in (("default", DEFAULT), ("pair", FORCE_PAIR)):
+            binding.regenvc_debug_set_phases(mask)
+            out = torch.full_like(q, float("nan"))
+            binding.regenvc_cross_attn_forward(q, k, v, out)
+            assert binding.regenvc_device_status() == 0
+            outs[name] = out
+    finally:
+        binding.regenvc_debug_set_phases(DEFAULT)
+    assert torch.equal(outs["default"], outs["pair"])
+    rows = torch.tensor([0, 1, 127, 128, 255, 256, 4095, 8192, 16000, 16383], device=dev)
+    heads = torch.tensor([0, h - 1], device=dev)
+    qs = q[rows][:, heads].cpu().contiguous()
+    ks, vs = k[:, heads].cpu().contiguous(), v[:, heads].cpu().contiguous()
+    ref = oracle.cross_attention(synth.bits(qs), synth.bits(ks), synth.bits(vs))
+    got = outs["pair"][rows][:, heads].double().cpu().numpy()
+    assert_parity(got, ref, float(vs.float().abs().max()), f"sampled rows, {h} heads")
+
+
 def test_debug_switch_argument_checks():
     L = binding.lib()
     assert L.regenvc_debug_set_phases(8) == binding.ERR_BAD_SHAPE           # neither pass selected
