@@ -41,8 +41,8 @@
 // staged (or written) and its Q buffer free.  Every load reads this GPU's own memory, every CTA fetches its own halves.
 //
 // Softmax keeps, per row, a reference m (log2 domain) and a row sum l.  m is set from the first tile's row
-// maximum (plus kRefMargin of headroom) and afterwards only raised when a probability would leave the fp16 range (p = 2^(s - m) > 65504).  As in
-// attn_pipelined.cu an item first runs optimistically (a thread only remembers a saturated partial sum).  A CTA that
+// maximum (plus kRefMargin of headroom) and afterwards only raised when a probability would leave the fp16 range
+// (p = 2^(s - m) > 65504).  As in attn_pipelined.cu an item first runs optimistically (a thread only remembers a saturated partial sum).  A CTA that
 // saw a saturation marks the item in a bit mask in its shared memory and carries on; after its last item the pair
 // meets at a cluster barrier, reads both CTAs' masks and runs the marked items again carefully (per-tile agreement
 // of a row group, row maximum, rescale of O, redo of the tile), overwriting what the optimistic run left.

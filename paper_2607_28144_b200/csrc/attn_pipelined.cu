@@ -18,8 +18,8 @@
 // of the finished output tile), then a ring of kStages 32 KB slots holding K'_0, V't_0, K'_1, ...
 //
 // Softmax keeps, per row, a reference m (log2 domain) and a row sum l.  m is set from the first tile's row
-// maximum (plus kRefMargin of headroom) and afterwards only raised when a probability would leave the fp16 range (p = 2^(s - m) > 65504),
-// so the probabilities of a tile are formed directly against the reference of the earlier tiles as soon as
+// maximum (plus kRefMargin of headroom) and afterwards only raised when a probability would leave the fp16 range
+// (p = 2^(s - m) > 65504), so the probabilities of a tile are formed directly against the reference of the earlier tiles as soon as
 // the scores arrive.  A saturated probability shows in the fp32 sum of its thread's part of the row.
 // The CTA first runs its key tiles OPTIMISTICALLY: every thread only remembers whether any of its sums
 // saturated, nothing is exchanged per tile (the per-tile agreement of the four warps that share 32 rows cost
