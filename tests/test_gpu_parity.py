@@ -235,6 +235,38 @@ def test_a_saturation_in_one_work_item_only(key):
     assert_parity(gpu[300:330, :1], ref[300:330, :1], float(v.float().abs().max()), "the saturated rows")
 
 
+@pytest.mark.parametrize("b", [18.0, 20.5, 21.5, 23.0, 26.0])
+@pytest.mark.parametrize("top_key", [5, 7000])
+def test_one_dominating_key_over_a_flat_tail_of_twelve_thousand(b, top_key):
+    """The worst case of the probabilities' fp16 floor: one key whose score lies `gap` log2 units above ALL the other
+    12479 keys (gap = 8 b log2(e) / sqrt(128): 18.4 to 26.5), with values of opposite sign, so that whatever weight of
+    the tail is lost shows up in full.  The kernels' softmax reference sits 4 log2 units above a row maximum: tail
+    probabilities from about 21 log2 units below the largest one on vanish from P.V.  The result must stay within
+    the stated error bound for every gap, wherever the dominating key comes (first tile or a late one)."""
+    n_q, n_kv, h = 256, 12480, 1
+    q = np.zeros((n_q, h, D), dtype=np.float32)
+    k = np.zeros((n_kv, h, D), dtype=np.float32)
+    v = -np.ones((n_kv, h, D), dtype=np.float32)
+    q[:, 0, 0] = 8.0
+    k[top_key, 0, 0] = b
+    v[top_key] = 1.0
+    rng = np.random.default_rng(71)
+    q[:, 0, 1:] = 0.01 * rng.standard_normal((n_q, D - 1))   # (rows differ a little; these do not touch the scores' gap)
+    q, k, v = synth.from_f32(q), synth.from_f32(k), synth.from_f32(v)
+    ref = oracle.cross_attention(synth.bits(q), synth.bits(k), synth.bits(v))
+    gap = 8.0 * b * np.log2(np.e) / np.sqrt(128.0)
+    tail = (n_kv - 1) * 2.0 ** -gap
+    np.testing.assert_allclose(ref[:, 0, 0], (1.0 - tail) / (1.0 + tail), rtol=1e-6)   # the oracle against the closed form
+    for bits in (3, 3 | 8):
+        binding.regenvc_debug_set_phases(bits)
+        try:
+            gpu = f64(run_gpu_cross(q, k, v))
+        finally:
+            binding.regenvc_debug_set_phases(3)
+        err = np.abs(gpu - ref).max()
+        assert err <= 1e-2, f"gap {gap:.1f} log2 units, kernel bits {bits}: max error {err:.2e} (tail weight {tail:.2e})"
+
+
 def test_heads_are_independent_on_the_gpu():
     T, H, W, h = 2, 9, 10, 4
     N = T * H * W
