@@ -271,6 +271,22 @@ def test_dominating_key_gives_that_value_row():
     np.testing.assert_allclose(o[2], v[13], rtol=0, atol=1e-12)
 
 
+@pytest.mark.parametrize("b", [2.0, 12.0, 23.0])
+def test_one_key_above_a_flat_tail_closed_form(b):
+    """q = 8 e_0; one key b e_0 with value +1, all 1999 others zero keys with value -1: the score gap is
+    8 b / sqrt(128) nats, the tail's weight t = 1999 exp(-gap), and every output element (1 - t) / (1 + t)."""
+    n_q, n_kv = 3, 2000
+    q = np.zeros((n_q, 1, 128), dtype=np.float32)
+    k = np.zeros((n_kv, 1, 128), dtype=np.float32)
+    v = -np.ones((n_kv, 1, 128), dtype=np.float32)
+    q[:, 0, 0] = 8.0
+    k[1234, 0, 0] = b
+    v[1234] = 1.0
+    out = oracle.cross_attention(synth.bits(synth.from_f32(q)), synth.bits(synth.from_f32(k)), synth.bits(synth.from_f32(v)))
+    t = (n_kv - 1) * math.exp(-8.0 * b / math.sqrt(128.0))
+    np.testing.assert_allclose(out, (1.0 - t) / (1.0 + t), rtol=1e-12, atol=1e-15)
+
+
 def test_core_equals_library_fp64_sdpa():
     rng = np.random.default_rng(10)
     q = rng.standard_normal((37, D)) * 1.5; k = rng.standard_normal((203, D)) * 1.5
